@@ -1,0 +1,110 @@
+// Internal declarations shared by the libsq translation units (host context + kernel launchers).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sq.h"
+
+namespace sq {
+
+constexpr int kMaxLayers = 256;
+constexpr int kMaxGroup = 128;          // query heads per KV head
+constexpr int kMinSplitTokens = 256;    // a split-K piece is never shorter than this
+constexpr int kTargetItems = 148 * 16;  // decode CTAs wanted per launch before split-K stops
+
+// Per-layer cache geometry, resident in device memory once the budgets are known.
+// k/v/pos/acc/victim offsets are BYTES from the pool base; logit_off counts floats from the
+// start of the logits area of the workspace.
+struct LayerDesc {
+  long long k_off, v_off, pos_off, acc_off, victim_off, logit_off;
+  int b;                  // budget: tokens kept per unit
+  int cap;                // slots per unit (b rounded up to page_tokens)
+  int b_heavy, b_recent;  // H2O split of b
+  int ring_base;          // Sliding Window 0, StreamingLLM n_sink: slots below it never rotate
+  int ring_origin;        // the position that maps to slot ring_base
+};
+
+// Slot of position x in a ring-managed (Sliding Window / StreamingLLM) cache.
+__host__ __device__ inline int ring_slot(int x, int b, int base, int origin) {
+  if (x < base) return x;
+  return base + (x - origin) % (b - base);
+}
+
+struct ImportanceArgs {
+  const void* a;
+  const void* b;
+  long long n_tok;
+  int hidden;
+  float* cta_partial;    // [n_cta]
+  unsigned int* ticket;  // zero on entry, zero again on exit
+  double* cos_sum;       // += sum over tokens of the cosine
+};
+
+struct AllocateArgs {
+  const double* cos_sum;
+  const long long* tok_count;
+  int n_layer, n_cluster;
+  long long b_init;
+  double p;
+  float* cos_sim;
+  int* budget;
+  unsigned char* is_g3;
+};
+
+struct GatherArgs {  // prompt rows -> cache slots of one layer
+  const void* k_prompt;
+  const void* v_prompt;
+  const float* acc_prompt;  // H2O, else null
+  char* pool;
+  LayerDesc ld;
+  int n_unit, prompt, n_keep, policy, head_dim;
+};
+
+struct ScoreArgs {  // H2O prompt scores of one layer
+  const void* q;
+  const void* k;
+  float* lse2;        // [B, Hq, P]  log2-domain row log-sum-exp
+  float* acc_prompt;  // [B, Hkv, P]
+  int batch, n_q_head, n_kv_head, prompt, head_dim;
+};
+
+struct DecodeArgs {
+  const LayerDesc* layers;
+  const int* order;  // layer indices sorted by budget, descending
+  char* pool;
+  float* logits;
+  float* part_stat;  // [item][group][2]   (max, sum) in the log2 domain
+  float* part_o;     // [item][group][head_dim]
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* out;
+  int* status;
+  int n_layer_total, layer_begin, layer_end;
+  int n_tok;  // tokens seen before this step == position of the new token
+  int batch, n_q_head, n_kv_head, head_dim, group;
+  int n_unit;  // batch * n_kv_head
+  int split_tokens, policy;
+  float scale_log2;  // log2(e) / sqrt(head_dim)
+};
+
+struct EvictArgs {
+  char* pool;
+  LayerDesc ld_old, ld_new;
+  int n_unit, len, n_tok, policy, n_sink, row_bytes;
+  int* status;
+};
+
+// Launchers: each returns the cudaError_t of its launches.
+cudaError_t launch_importance(const ImportanceArgs& a, int dtype, int n_cta, cudaStream_t s);
+cudaError_t launch_allocate(const AllocateArgs& a, cudaStream_t s);
+cudaError_t launch_gather(const GatherArgs& a, int dtype, cudaStream_t s);
+cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, cudaStream_t s);
+cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc& ld, char* pool,
+                                 cudaStream_t s);
+cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int len, int next_pos, cudaStream_t s);
+cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, cudaStream_t s);
+cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s);
+
+}  // namespace sq
