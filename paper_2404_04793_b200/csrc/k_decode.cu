@@ -1,0 +1,369 @@
+// Decode step of Algorithm 1 (steps 15-22) for a range of layers in one launch: append the new
+// token into the slot C_seq frees, attend over the kept slots (split-K flash-decode, all query
+// heads of a KV head share one pass over K/V), and for H2O add the received probabilities to
+// the per-token scores and choose the slot the next append will reuse.
+#include "sq_device.cuh"
+#include "sq_internal.h"
+#include "sq_select.cuh"
+
+namespace sq {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+struct ItemLoc {
+  int layer, local, n_split, base;
+};
+
+__device__ __forceinline__ int n_split_of(const DecodeArgs& a, int b) {
+  int len = min(a.n_tok + 1, b);
+  return (len + a.split_tokens - 1) / a.split_tokens;
+}
+
+// Work items of a launch are numbered layer by layer in `order` (largest budget first), and
+// within a layer as unit * n_split + split.  Each warp finds, by a prefix scan over the
+// layers, either the layer an item index falls in (want_layer < 0) or the first item of a
+// given layer.
+__device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_layer, ItemLoc& out) {
+  const int lane = threadIdx.x & 31;
+  int running = 0;
+  for (int c = 0; c < a.n_layer_total; c += 32) {
+    const int i = c + lane;
+    int l = -1, ns = 0, cnt = 0;
+    if (i < a.n_layer_total) {
+      int li = a.order[i];
+      if (li >= a.layer_begin && li < a.layer_end) {
+        l = li;
+        ns = n_split_of(a, a.layers[li].b);
+        cnt = a.n_unit * ns;
+      }
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(kFull, incl, o);
+      if (lane >= o) incl += t;
+    }
+    unsigned hit = (want_layer >= 0) ? __ballot_sync(kFull, l == want_layer)
+                                     : __ballot_sync(kFull, cnt > 0 && idx < running + incl);
+    if (hit) {
+      const int src = __ffs(hit) - 1;
+      out.layer = __shfl_sync(kFull, l, src);
+      out.n_split = __shfl_sync(kFull, ns, src);
+      out.base = running + __shfl_sync(kFull, incl - cnt, src);
+      out.local = idx - out.base;
+      return true;
+    }
+    running += __shfl_sync(kFull, incl, 31);
+  }
+  return false;
+}
+
+// One CTA (4 warps) per (layer, unit, split).  A K or V row is D*sizeof(T) bytes = LPR lanes
+// x 16 bytes, so a warp reads 32/LPR consecutive rows per load instruction, fully coalesced.
+// Each lane keeps its 16-byte slice of up to GT query heads (pre-scaled by log2(e)/sqrt(d))
+// and of their output accumulators in fp32; logits are reduced over the LPR lanes by
+// shuffles, and the softmax runs online in the log2 domain over batches of U rows.
+template <typename T, int D, int GT>
+__global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;   // lanes per row
+  constexpr int RPW = 32 / LPR;  // rows per warp per load
+  constexpr int U = 4;           // rows in flight per lane
+  __shared__ float sm_o[4][GT][D];
+  __shared__ float sm_m[4][GT], sm_l[4][GT];
+
+  ItemLoc it;
+  if (!locate(a, blockIdx.x, -1, it)) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane % LPR, rg = lane / LPR;
+  const LayerDesc* ldp = a.layers + it.layer;
+  const int b = ldp->b, cap = ldp->cap;
+  const int unit = it.local / it.n_split, split = it.local - unit * it.n_split;
+  const int len = min(a.n_tok + 1, b);
+  const bool h2o = (a.policy == SQ_POLICY_H2O);
+  int w;  // slot that receives the new token
+  if (h2o) {
+    w = (a.n_tok < b) ? a.n_tok : reinterpret_cast<const int*>(a.pool + ldp->victim_off)[unit];
+    if (w < 0 || w >= b) {
+      if (tid == 0) atomicOr(a.status, 2);
+      w = 0;
+    }
+  } else {
+    w = ring_slot(a.n_tok, b, ldp->ring_base, ldp->ring_origin);
+  }
+  const int t0 = split * a.split_tokens, t1 = min(len, t0 + a.split_tokens);
+  const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
+  const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
+  const T* Kb = reinterpret_cast<const T*>(a.pool + ldp->k_off) + (size_t)unit * cap * D;
+  const T* Vb = reinterpret_cast<const T*>(a.pool + ldp->v_off) + (size_t)unit * cap * D;
+  const T* qb = reinterpret_cast<const T*>(a.q) + (tok * a.n_q_head + (size_t)kvh * a.group) * D;
+  const T* kn = reinterpret_cast<const T*>(a.k_new) + (tok * a.n_kv_head + kvh) * D;
+  const T* vn = reinterpret_cast<const T*>(a.v_new) + (tok * a.n_kv_head + kvh) * D;
+  T* ob = reinterpret_cast<T*>(a.out) + (tok * a.n_q_head + (size_t)kvh * a.group) * D;
+  float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * a.group;  // [slot][group]
+  float* stat = a.part_stat + (size_t)blockIdx.x * a.group * 2;
+  float* po = a.part_o + (size_t)blockIdx.x * a.group * D;
+
+  for (int hb = 0; hb < a.group; hb += GT) {
+    float qr[GT][EPV], o[GT][EPV], m[GT], l[GT];
+#pragma unroll
+    for (int g = 0; g < GT; ++g) {
+      m[g] = -INFINITY;
+      l[g] = 0.f;
+      if (hb + g < a.group) {
+        widen<T>(ld_stream(qb + (size_t)(hb + g) * D + sub * EPV), qr[g]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) qr[g][e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) {
+        qr[g][e] *= a.scale_log2;
+        o[g][e] = 0.f;
+      }
+    }
+    for (int r0 = t0 + warp * (U * RPW); r0 < t1; r0 += 4 * U * RPW) {
+      uint4 kq[U], vq[U];
+      bool ok[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int row = r0 + u * RPW + rg;
+        ok[u] = row < t1;
+        const int rr = ok[u] ? row : t0;
+        const T* kp = (rr == w) ? kn : Kb + (size_t)rr * D;
+        const T* vp = (rr == w) ? vn : Vb + (size_t)rr * D;
+        kq[u] = ld_stream(kp + sub * EPV);
+        vq[u] = ld_stream(vp + sub * EPV);
+      }
+      float s[U][GT];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float kf[EPV];
+        widen<T>(kq[u], kf);
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          float d = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) d = fmaf(qr[g][e], kf[e], d);
+#pragma unroll
+          for (int off = LPR / 2; off > 0; off >>= 1) d += __shfl_xor_sync(kFull, d, off);
+          s[u][g] = ok[u] ? d : -INFINITY;
+        }
+      }
+      if (h2o) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (!ok[u]) continue;
+          const int row = r0 + u * RPW + rg;
+#pragma unroll
+          for (int g = 0; g < GT; ++g)
+            if (sub == g && hb + g < a.group) logit[(size_t)row * a.group + hb + g] = s[u][g];
+        }
+      }
+      float mn[GT];
+#pragma unroll
+      for (int g = 0; g < GT; ++g) {
+        float mx = s[0][g];
+#pragma unroll
+        for (int u = 1; u < U; ++u) mx = fmaxf(mx, s[u][g]);
+        mn[g] = fmaxf(m[g], mx);
+        if (mn[g] > -INFINITY) {
+          const float corr = exp2f(m[g] - mn[g]);
+          l[g] *= corr;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) o[g][e] *= corr;
+          m[g] = mn[g];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float vf[EPV];
+        widen<T>(vq[u], vf);
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          const float p = (s[u][g] > -INFINITY) ? exp2f(s[u][g] - mn[g]) : 0.f;
+          l[g] += p;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) o[g][e] = fmaf(p, vf[e], o[g][e]);
+        }
+      }
+    }
+    // merge the row groups of the warp
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+      for (int g = 0; g < GT; ++g) {
+        const float m2 = __shfl_xor_sync(kFull, m[g], off);
+        const float l2 = __shfl_xor_sync(kFull, l[g], off);
+        const float mx = fmaxf(m[g], m2);
+        const float f1 = (m[g] > -INFINITY) ? exp2f(m[g] - mx) : 0.f;
+        const float f2 = (m2 > -INFINITY) ? exp2f(m2 - mx) : 0.f;
+        l[g] = l[g] * f1 + l2 * f2;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+          const float o2 = __shfl_xor_sync(kFull, o[g][e], off);
+          o[g][e] = o[g][e] * f1 + o2 * f2;
+        }
+        m[g] = mx;
+      }
+    }
+    if (rg == 0) {
+#pragma unroll
+      for (int g = 0; g < GT; ++g) {
+        if (sub == 0) {
+          sm_m[warp][g] = m[g];
+          sm_l[warp][g] = l[g];
+        }
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) sm_o[warp][g][sub * EPV + e] = o[g][e];
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < GT * D; idx += 128) {
+      const int g = idx / D, e = idx - g * D, h = hb + g;
+      if (h >= a.group) continue;
+      float M = -INFINITY;
+#pragma unroll
+      for (int ww = 0; ww < 4; ++ww) M = fmaxf(M, sm_m[ww][g]);
+      float L = 0.f, O = 0.f;
+#pragma unroll
+      for (int ww = 0; ww < 4; ++ww) {
+        const float mw = sm_m[ww][g];
+        const float f = (mw > -INFINITY) ? exp2f(mw - M) : 0.f;
+        L += sm_l[ww][g] * f;
+        O += sm_o[ww][g][e] * f;
+      }
+      if (it.n_split == 1)
+        ob[(size_t)h * D + e] = narrow<T>(O / L);
+      else
+        po[(size_t)h * D + e] = O;
+      if (e == 0) {
+        stat[h * 2] = M;
+        stat[h * 2 + 1] = L;
+      }
+    }
+    __syncthreads();
+  }
+
+  // the CTA whose range holds slot w stores the new token (nobody reads that slot this step)
+  if (w >= t0 && w < t1) {
+    if (tid < 2 * LPR) {
+      const bool is_v = tid >= LPR;
+      const int v = is_v ? tid - LPR : tid;
+      const T* src = (is_v ? vn : kn) + v * EPV;
+      T* dst = const_cast<T*>(is_v ? Vb : Kb) + (size_t)w * D + v * EPV;
+      *reinterpret_cast<uint4*>(dst) = ld_stream(src);
+    }
+    if (tid == 64) {
+      reinterpret_cast<int*>(a.pool + ldp->pos_off)[(size_t)unit * cap + w] = a.n_tok;
+      if (h2o) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
+    }
+  }
+}
+
+// One CTA per (layer, unit): merges the split-K partials into the output and, for H2O, adds
+// each kept token's probabilities (summed over the group's heads in head order) to its score
+// and picks the slot the next append replaces.
+template <typename T>
+__global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
+  __shared__ SelScratch sc;
+  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup];
+  const int n_layers = a.layer_end - a.layer_begin;
+  const int layer = a.layer_begin + blockIdx.x / a.n_unit;
+  const int unit = blockIdx.x % a.n_unit;
+  (void)n_layers;
+  ItemLoc it;
+  if (!locate(a, 0, layer, it)) return;
+  const int tid = threadIdx.x, D = a.head_dim, G = a.group, ns = it.n_split;
+  const LayerDesc* ldp = a.layers + layer;
+  const int b = ldp->b, cap = ldp->cap;
+  const size_t item0 = (size_t)it.base + (size_t)unit * ns;
+  const float* stat = a.part_stat + item0 * G * 2;
+  for (int h = tid; h < G; h += kSelThreads) {
+    float M = -INFINITY;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, stat[((size_t)s * G + h) * 2]);
+    float L = 0.f;
+    for (int s = 0; s < ns; ++s) {
+      const float ms = stat[((size_t)s * G + h) * 2];
+      L += stat[((size_t)s * G + h) * 2 + 1] * ((ms > -INFINITY) ? exp2f(ms - M) : 0.f);
+    }
+    s_M[h] = M;
+    s_invL[h] = 1.f / L;
+  }
+  __syncthreads();
+  if (ns > 1) {
+    const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
+    const size_t tok = (size_t)(layer - a.layer_begin) * a.batch + seq;
+    T* ob = reinterpret_cast<T*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * D;
+    const float* po = a.part_o + item0 * G * D;
+    for (int idx = tid; idx < G * D; idx += kSelThreads) {
+      const int h = idx / D;
+      float O = 0.f;
+      for (int s = 0; s < ns; ++s) {
+        const float ms = stat[((size_t)s * G + h) * 2];
+        O += po[(size_t)s * G * D + idx] * ((ms > -INFINITY) ? exp2f(ms - s_M[h]) : 0.f);
+      }
+      ob[idx] = narrow<T>(O * s_invL[h]);
+    }
+  }
+  if (a.policy != SQ_POLICY_H2O) return;
+  const int len = min(a.n_tok + 1, b);
+  const bool full = (len == b);
+  const int thr = a.n_tok + 1 - ldp->b_recent;  // next step: positions <= thr are outside the recent window
+  const int* pos = reinterpret_cast<const int*>(a.pool + ldp->pos_off) + (size_t)unit * cap;
+  float* acc = reinterpret_cast<float*>(a.pool + ldp->acc_off) + (size_t)unit * cap;
+  const float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  unsigned long long best = ~0ull;
+  int best_slot = -1;
+  for (int slot = tid; slot < len; slot += kSelThreads) {
+    float gain = 0.f;
+    for (int h = 0; h < G; ++h) gain += exp2f(logit[(size_t)slot * G + h] - s_M[h]) * s_invL[h];
+    const float v = acc[slot] + gain;
+    acc[slot] = v;
+    if (full) {
+      const int p = pos[slot];
+      if (p <= thr) {
+        const unsigned long long r = victim_rank(v, p);
+        if (r < best) {
+          best = r;
+          best_slot = slot;
+        }
+      }
+    }
+  }
+  if (full) {
+    best_slot = block_argmin(sc, best, best_slot);
+    if (tid == 0) reinterpret_cast<int*>(a.pool + ldp->victim_off)[unit] = best_slot;
+  }
+}
+
+template <typename T, int D>
+static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
+  if (a.group == 1)
+    decode_attn_kernel<T, D, 1><<<n_items, 128, 0, s>>>(a);
+  else if (a.group <= 4)
+    decode_attn_kernel<T, D, 4><<<n_items, 128, 0, s>>>(a);
+  else
+    decode_attn_kernel<T, D, 8><<<n_items, 128, 0, s>>>(a);
+}
+
+cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, cudaStream_t s) {
+  if (n_items <= 0) return cudaSuccess;
+  if (dtype == SQ_F32) {
+    if (a.head_dim == 64) launch_attn_g<float, 64>(a, n_items, s);
+    else launch_attn_g<float, 128>(a, n_items, s);
+  } else {
+    if (a.head_dim == 64) launch_attn_g<__nv_bfloat16, 64>(a, n_items, s);
+    else launch_attn_g<__nv_bfloat16, 128>(a, n_items, s);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || !need_combine) return e;
+  const int n_cta = (a.layer_end - a.layer_begin) * a.n_unit;
+  if (dtype == SQ_F32)
+    decode_combine_kernel<float><<<n_cta, kSelThreads, 0, s>>>(a);
+  else
+    decode_combine_kernel<__nv_bfloat16><<<n_cta, kSelThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace sq

@@ -1,0 +1,658 @@
+// Host side of libsq: context, memory layout of the caller's pool and workspace, argument
+// validation, call-order checks and kernel launches.  See include/sq.h for the contract.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "sq_internal.h"
+
+using namespace sq;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int elem_bytes(int dtype) { return dtype == SQ_F32 ? 4 : 2; }
+constexpr int kMaxImportanceCtas = 4096;
+
+struct WsLayout {
+  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, layers, order;
+  size_t part_stat, part_o, logits, acc_prompt, lse2, total;
+  size_t items_cap, logits_floats;
+};
+
+struct HostStage {  // pinned
+  int32_t budget[kMaxLayers];
+  uint8_t is_g3[kMaxLayers];
+  float cos_sim[kMaxLayers];
+  long long tok_count[kMaxLayers];
+  LayerDesc layers[kMaxLayers];
+  int order[kMaxLayers];
+  int32_t status;
+};
+
+}  // namespace
+
+struct sq_ctx {
+  sq_config cfg;
+  int64_t b_init_cap;
+  char* pool;
+  size_t pool_bytes;
+  char* ws;
+  size_t ws_bytes;
+  WsLayout wl;
+  HostStage* hs;
+  cudaEvent_t ev;
+  int n_sm;
+  int batch, prompt;
+  bool begun;
+  int budget_state;  // 0 none, 1 computed on device (copy in flight), 2 on host, laid out
+  int n_tok[kMaxLayers];
+  bool prefilled[kMaxLayers];
+  bool importance_seen[kMaxLayers];
+  std::string err;
+};
+
+namespace {
+
+int fail(sq_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  return code;
+}
+
+int check_config(const sq_config* c, std::string* why) {
+  auto bad = [&](const char* m) {
+    if (why) *why = m;
+    return (int)SQ_ERR_INVALID_ARG;
+  };
+  if (!c) return bad("config is NULL");
+  if (c->n_layer < 1 || c->n_layer > kMaxLayers) return bad("n_layer must be in 1..256");
+  if (c->n_kv_head < 1 || c->n_q_head < 1 || c->n_q_head % c->n_kv_head) return bad("n_q_head must be a multiple of n_kv_head");
+  if (c->n_q_head / c->n_kv_head > kMaxGroup) return bad("more than 128 query heads per KV head");
+  if (c->head_dim != 64 && c->head_dim != 128) {
+    if (why) *why = "head_dim must be 64 or 128";
+    return (int)SQ_ERR_UNSUPPORTED;
+  }
+  if (c->hidden < 8 || c->hidden % 8) return bad("hidden must be a positive multiple of 8");
+  if (c->max_batch < 1 || c->max_prompt < 1 || c->max_new_tokens < 0) return bad("max_batch/max_prompt/max_new_tokens");
+  if (c->dtype != SQ_F32 && c->dtype != SQ_BF16) return bad("dtype");
+  if (c->policy < SQ_POLICY_SLIDING_WINDOW || c->policy > SQ_POLICY_H2O) return bad("policy");
+  if (c->policy == SQ_POLICY_STREAMING_LLM && c->n_sink < 0) return bad("n_sink");
+  if (c->policy == SQ_POLICY_H2O && (c->heavy_den < 1 || c->heavy_num < 0 || c->heavy_num >= c->heavy_den))
+    return bad("H2O needs 0 <= heavy_num < heavy_den");
+  if (c->n_cluster != 2 && c->n_cluster != 3) return bad("n_cluster must be 2 or 3");
+  if (c->page_tokens < 1) return bad("page_tokens must be >= 1");
+  return SQ_OK;
+}
+
+size_t pool_bytes_for(const sq_config& c, int64_t b_init) {
+  const size_t U = (size_t)c.max_batch * c.n_kv_head;
+  const size_t tokens = (size_t)c.n_layer * (size_t)b_init + (size_t)c.n_layer * (c.page_tokens - 1);
+  size_t per_tok = 2 * (size_t)c.head_dim * elem_bytes(c.dtype) + 4 + (c.policy == SQ_POLICY_H2O ? 4 : 0);
+  return U * tokens * per_tok + (size_t)c.n_layer * (U * 4 + 6 * kAlign);
+}
+
+WsLayout ws_layout(const sq_config& c, int64_t b_init) {
+  WsLayout w{};
+  const size_t L = c.n_layer, U = (size_t)c.max_batch * c.n_kv_head, G = c.n_q_head / c.n_kv_head;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes);
+    return o;
+  };
+  w.cos_sum = take(8 * L);
+  w.tok_count = take(8 * L);
+  w.cta_partial = take(4 * (size_t)kMaxImportanceCtas);
+  w.ticket = take(4);
+  w.cos_sim = take(4 * L);
+  w.budget = take(4 * L);
+  w.is_g3 = take(L);
+  w.status = take(4);
+  w.layers = take(sizeof(LayerDesc) * L);
+  w.order = take(4 * L);
+  w.items_cap = (size_t)kTargetItems + U * L;
+  w.part_stat = take(w.items_cap * G * 2 * 4);
+  w.part_o = take(w.items_cap * G * c.head_dim * 4);
+  const bool h2o = c.policy == SQ_POLICY_H2O;
+  w.logits_floats = h2o ? U * G * (L * (size_t)b_init + L * (c.page_tokens - 1)) : 0;
+  w.logits = take(w.logits_floats * 4);
+  w.acc_prompt = take(h2o ? U * (size_t)c.max_prompt * 4 : 0);
+  w.lse2 = take(h2o ? (size_t)c.max_batch * c.n_q_head * c.max_prompt * 4 : 0);
+  w.total = off;
+  return w;
+}
+
+template <typename T>
+T* ws_ptr(sq_ctx* c, size_t off) {
+  return reinterpret_cast<T*>(c->ws + off);
+}
+
+#define SQ_CUDA(c, expr)                                                                         \
+  do {                                                                                           \
+    cudaError_t e__ = (expr);                                                                    \
+    if (e__ != cudaSuccess)                                                                      \
+      return fail((c), SQ_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__));        \
+  } while (0)
+
+// Computes the per-layer cache geometry for the budgets in hs->budget and uploads it.
+int build_layout(sq_ctx* c, cudaStream_t st) {
+  const sq_config& cfg = c->cfg;
+  const size_t U = (size_t)c->batch * cfg.n_kv_head, G = cfg.n_q_head / cfg.n_kv_head;
+  const size_t row = (size_t)cfg.head_dim * elem_bytes(cfg.dtype);
+  const bool h2o = cfg.policy == SQ_POLICY_H2O;
+  size_t off = 0, lfl = 0;
+  for (int l = 0; l < cfg.n_layer; ++l) {
+    LayerDesc& d = c->hs->layers[l];
+    const int b = c->hs->budget[l];
+    if (b < 1) return fail(c, SQ_ERR_INVALID_ARG, "a layer budget is below 1");
+    if (cfg.policy == SQ_POLICY_STREAMING_LLM && b <= cfg.n_sink)
+      return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
+    d.b = b;
+    d.cap = (b + cfg.page_tokens - 1) / cfg.page_tokens * cfg.page_tokens;
+    d.b_heavy = h2o ? (int)(((long long)b * cfg.heavy_num) / cfg.heavy_den) : 0;
+    d.b_recent = b - d.b_heavy;
+    d.ring_base = (cfg.policy == SQ_POLICY_STREAMING_LLM) ? cfg.n_sink : 0;
+    d.ring_origin = std::max(d.ring_base, c->prompt - (b - d.ring_base));
+    d.k_off = (long long)off;
+    off = align_up(off + U * d.cap * row);
+    d.v_off = (long long)off;
+    off = align_up(off + U * d.cap * row);
+    d.pos_off = (long long)off;
+    off = align_up(off + U * d.cap * 4);
+    d.acc_off = (long long)off;
+    if (h2o) off = align_up(off + U * d.cap * 4);
+    d.victim_off = (long long)off;
+    off = align_up(off + U * 4);
+    d.logit_off = (long long)lfl;
+    if (h2o) lfl += U * d.cap * G;
+  }
+  if (off > c->pool_bytes) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the cache pool");
+  if (lfl > c->wl.logits_floats) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the workspace");
+  std::vector<int> ord(cfg.n_layer);
+  for (int l = 0; l < cfg.n_layer; ++l) ord[l] = l;
+  std::stable_sort(ord.begin(), ord.end(), [&](int x, int y) { return c->hs->budget[x] > c->hs->budget[y]; });
+  std::copy(ord.begin(), ord.end(), c->hs->order);
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers), c->hs->layers, sizeof(LayerDesc) * cfg.n_layer,
+                             cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs->order, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
+  // the staging block is reused by later calls: make sure the copies have left it
+  SQ_CUDA(c, cudaStreamSynchronize(st));
+  c->budget_state = 2;
+  return SQ_OK;
+}
+
+int ensure_budgets(sq_ctx* c, cudaStream_t st) {
+  if (c->budget_state == 2) return SQ_OK;
+  if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "budgets not set: call sq_allocate_budgets or sq_set_budgets first");
+  SQ_CUDA(c, cudaEventSynchronize(c->ev));
+  return build_layout(c, st);
+}
+
+int upload_layer(sq_ctx* c, int l, cudaStream_t st) {
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers) + l, &c->hs->layers[l], sizeof(LayerDesc),
+                             cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaStreamSynchronize(st));
+  return SQ_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int sq_query_sizes(const sq_config* cfg, int64_t b_init, size_t* pool_bytes, size_t* workspace_bytes) {
+  int rc = check_config(cfg, nullptr);
+  if (rc != SQ_OK) return rc;
+  if (b_init < 1 || !pool_bytes || !workspace_bytes) return SQ_ERR_INVALID_ARG;
+  *pool_bytes = pool_bytes_for(*cfg, b_init);
+  *workspace_bytes = ws_layout(*cfg, b_init).total;
+  return SQ_OK;
+}
+
+int sq_ctx_create(const sq_config* cfg, int64_t b_init, void* pool, size_t pool_bytes, void* workspace,
+                  size_t workspace_bytes, sq_ctx** out) {
+  if (!out) return SQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg, nullptr);
+  if (rc != SQ_OK) return rc;
+  if (b_init < 1 || !pool || !workspace) return SQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(pool) % kAlign) || (reinterpret_cast<uintptr_t>(workspace) % kAlign))
+    return SQ_ERR_INVALID_ARG;
+  if (pool_bytes < pool_bytes_for(*cfg, b_init)) return SQ_ERR_CAPACITY;
+  WsLayout wl = ws_layout(*cfg, b_init);
+  if (workspace_bytes < wl.total) return SQ_ERR_CAPACITY;
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SQ_ERR_CUDA;
+  sq_ctx* c = new (std::nothrow) sq_ctx();
+  if (!c) return SQ_ERR_CAPACITY;
+  c->cfg = *cfg;
+  c->b_init_cap = b_init;
+  c->pool = static_cast<char*>(pool);
+  c->pool_bytes = pool_bytes;
+  c->ws = static_cast<char*>(workspace);
+  c->ws_bytes = workspace_bytes;
+  c->wl = wl;
+  c->n_sm = n_sm;
+  c->begun = false;
+  c->budget_state = 0;
+  c->hs = nullptr;
+  if (cudaHostAlloc(reinterpret_cast<void**>(&c->hs), sizeof(HostStage), cudaHostAllocDefault) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev, cudaEventDisableTiming) != cudaSuccess) {
+    if (c->hs) cudaFreeHost(c->hs);
+    delete c;
+    return SQ_ERR_CUDA;
+  }
+  std::memset(c->hs, 0, sizeof(HostStage));
+  *out = c;
+  return SQ_OK;
+}
+
+int sq_ctx_destroy(sq_ctx* c) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaEventDestroy(c->ev);
+  cudaFreeHost(c->hs);
+  delete c;
+  return SQ_OK;
+}
+
+const char* sq_last_error(sq_ctx* c) { return c ? c->err.c_str() : "context is NULL"; }
+
+int sq_begin_sequence_batch(sq_ctx* c, int32_t batch, int32_t prompt_len, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (batch < 1 || batch > c->cfg.max_batch) return fail(c, SQ_ERR_INVALID_ARG, "batch out of range");
+  if (prompt_len < 1 || prompt_len > c->cfg.max_prompt) return fail(c, SQ_ERR_INVALID_ARG, "prompt_len out of range");
+  c->batch = batch;
+  c->prompt = prompt_len;
+  c->begun = true;
+  c->budget_state = 0;
+  for (int l = 0; l < c->cfg.n_layer; ++l) {
+    c->n_tok[l] = 0;
+    c->prefilled[l] = false;
+    c->importance_seen[l] = false;
+    c->hs->tok_count[l] = 0;
+  }
+  // everything up to the layer table: statistics, ticket, budgets, status
+  SQ_CUDA(c, cudaMemsetAsync(c->ws, 0, c->wl.layers, st));
+  return SQ_OK;
+}
+
+int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const void* hidden_out, int64_t n_tok_total,
+                        void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (layer < 0 || layer >= c->cfg.n_layer) return fail(c, SQ_ERR_INVALID_ARG, "layer out of range");
+  if (!hidden_in || !hidden_out || !aligned16(hidden_in) || !aligned16(hidden_out))
+    return fail(c, SQ_ERR_INVALID_ARG, "hidden state pointers must be non-NULL and 16-byte aligned");
+  if (n_tok_total < 0) return fail(c, SQ_ERR_INVALID_ARG, "n_tok_total is negative");
+  if (n_tok_total == 0) return SQ_OK;
+  ImportanceArgs a;
+  a.a = hidden_in;
+  a.b = hidden_out;
+  a.n_tok = n_tok_total;
+  a.hidden = c->cfg.hidden;
+  a.cta_partial = ws_ptr<float>(c, c->wl.cta_partial);
+  a.ticket = ws_ptr<unsigned int>(c, c->wl.ticket);
+  a.cos_sum = ws_ptr<double>(c, c->wl.cos_sum) + layer;
+  long long want = (n_tok_total + 7) / 8;
+  int n_cta = (int)std::min<long long>(want, std::min(kMaxImportanceCtas, c->n_sm * 8));
+  SQ_CUDA(c, launch_importance(a, c->cfg.dtype, n_cta, static_cast<cudaStream_t>(stream)));
+  c->hs->tok_count[layer] += n_tok_total;
+  c->importance_seen[layer] = true;
+  return SQ_OK;
+}
+
+int sq_allocate_budgets(sq_ctx* c, int64_t b_init, double p, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (!(p > 0.0 && p <= 1.0)) return fail(c, SQ_ERR_INVALID_ARG, "p must satisfy 0 < p <= 1");
+  if (b_init < 1 || b_init > c->b_init_cap) return fail(c, SQ_ERR_INVALID_ARG, "b_init must be in 1..the context's b_init");
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    if (!c->importance_seen[l]) return fail(c, SQ_ERR_STATE, "sq_layer_importance has not been called for every layer");
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<long long>(c, c->wl.tok_count), c->hs->tok_count, 8 * c->cfg.n_layer,
+                             cudaMemcpyHostToDevice, st));
+  AllocateArgs a;
+  a.cos_sum = ws_ptr<double>(c, c->wl.cos_sum);
+  a.tok_count = ws_ptr<long long>(c, c->wl.tok_count);
+  a.n_layer = c->cfg.n_layer;
+  a.n_cluster = c->cfg.n_cluster;
+  a.b_init = b_init;
+  a.p = p;
+  a.cos_sim = ws_ptr<float>(c, c->wl.cos_sim);
+  a.budget = ws_ptr<int>(c, c->wl.budget);
+  a.is_g3 = ws_ptr<unsigned char>(c, c->wl.is_g3);
+  SQ_CUDA(c, launch_allocate(a, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs->budget, a.budget, 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs->is_g3, a.is_g3, c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs->cos_sim, a.cos_sim, 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaEventRecord(c->ev, st));
+  c->budget_state = 1;
+  for (int l = 0; l < c->cfg.n_layer; ++l) c->prefilled[l] = false;
+  return SQ_OK;
+}
+
+int sq_set_budgets(sq_ctx* c, const int32_t* budgets_host, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (!budgets_host) return fail(c, SQ_ERR_INVALID_ARG, "budgets_host is NULL");
+  if (c->budget_state == 1) SQ_CUDA(c, cudaEventSynchronize(c->ev));
+  for (int l = 0; l < c->cfg.n_layer; ++l) {
+    c->hs->budget[l] = budgets_host[l];
+    c->hs->is_g3[l] = 0;
+    c->prefilled[l] = false;
+  }
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs->budget, 4 * c->cfg.n_layer, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemsetAsync(ws_ptr<unsigned char>(c, c->wl.is_g3), 0, c->cfg.n_layer, st));
+  c->budget_state = 0;
+  int rc = build_layout(c, st);
+  return rc;
+}
+
+int sq_prefill_compress(sq_ctx* c, int32_t layer, const void* k_prompt, const void* v_prompt, const void* q_prompt,
+                        const float* acc_prompt, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (layer < 0 || layer >= c->cfg.n_layer) return fail(c, SQ_ERR_INVALID_ARG, "layer out of range");
+  if (!k_prompt || !v_prompt || !aligned16(k_prompt) || !aligned16(v_prompt))
+    return fail(c, SQ_ERR_INVALID_ARG, "k_prompt/v_prompt must be non-NULL and 16-byte aligned");
+  const bool h2o = c->cfg.policy == SQ_POLICY_H2O;
+  if (h2o && !q_prompt && !acc_prompt) return fail(c, SQ_ERR_INVALID_ARG, "H2O needs q_prompt or acc_prompt");
+  int rc = ensure_budgets(c, st);
+  if (rc != SQ_OK) return rc;
+  const LayerDesc& ld = c->hs->layers[layer];
+  const int U = c->batch * c->cfg.n_kv_head, P = c->prompt;
+  const int n_keep = std::min(P, ld.b);
+  const float* acc = nullptr;
+  if (h2o) {
+    if (acc_prompt) {
+      acc = acc_prompt;
+    } else {
+      ScoreArgs s;
+      s.q = q_prompt;
+      s.k = k_prompt;
+      s.lse2 = ws_ptr<float>(c, c->wl.lse2);
+      s.acc_prompt = ws_ptr<float>(c, c->wl.acc_prompt);
+      s.batch = c->batch;
+      s.n_q_head = c->cfg.n_q_head;
+      s.n_kv_head = c->cfg.n_kv_head;
+      s.prompt = P;
+      s.head_dim = c->cfg.head_dim;
+      SQ_CUDA(c, launch_prefill_scores(s, c->cfg.dtype, st));
+      acc = s.acc_prompt;
+    }
+    SQ_CUDA(c, launch_select_prompt(acc, U, P, ld, c->pool, st));
+  }
+  GatherArgs g;
+  g.k_prompt = k_prompt;
+  g.v_prompt = v_prompt;
+  g.acc_prompt = acc;
+  g.pool = c->pool;
+  g.ld = ld;
+  g.n_unit = U;
+  g.prompt = P;
+  g.n_keep = n_keep;
+  g.policy = c->cfg.policy;
+  g.head_dim = c->cfg.head_dim;
+  SQ_CUDA(c, launch_gather(g, c->cfg.dtype, st));
+  if (h2o && n_keep == ld.b) SQ_CUDA(c, launch_pick_victim(c->pool, ld, U, n_keep, P, st));
+  c->n_tok[layer] = P;
+  c->prefilled[layer] = true;
+  return SQ_OK;
+}
+
+int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void* q, const void* k_new,
+                   const void* v_new, void* out, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (layer_begin < 0 || layer_end > c->cfg.n_layer || layer_begin >= layer_end)
+    return fail(c, SQ_ERR_INVALID_ARG, "layer range");
+  if (!q || !k_new || !v_new || !out || !aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out))
+    return fail(c, SQ_ERR_INVALID_ARG, "q/k_new/v_new/out must be non-NULL and 16-byte aligned");
+  int rc = ensure_budgets(c, st);
+  if (rc != SQ_OK) return rc;
+  const sq_config& cfg = c->cfg;
+  for (int l = layer_begin; l < layer_end; ++l) {
+    if (!c->prefilled[l]) return fail(c, SQ_ERR_STATE, "sq_prefill_compress has not been called for a layer in the range");
+    if (c->n_tok[l] >= cfg.max_prompt + cfg.max_new_tokens) return fail(c, SQ_ERR_CAPACITY, "max_new_tokens exceeded");
+  }
+  const int U = c->batch * cfg.n_kv_head, G = cfg.n_q_head / cfg.n_kv_head;
+  const size_t eb = elem_bytes(cfg.dtype);
+  const size_t q_layer = (size_t)c->batch * cfg.n_q_head * cfg.head_dim * eb;
+  const size_t kv_layer = (size_t)c->batch * cfg.n_kv_head * cfg.head_dim * eb;
+  int s = layer_begin;
+  while (s < layer_end) {
+    int e = s + 1;
+    while (e < layer_end && c->n_tok[e] == c->n_tok[s]) ++e;
+    const int n_tok = c->n_tok[s];
+    long long total = 0;
+    for (int l = s; l < e; ++l) total += (long long)U * std::min(n_tok + 1, c->hs->layers[l].b);
+    int split = 1 << 30;
+    if ((long long)U * (e - s) < kTargetItems / 2)
+      split = (int)std::max<long long>(kMinSplitTokens, (total + kTargetItems - 1) / kTargetItems);
+    long long n_items = 0;
+    bool any_split = false;
+    for (int l = s; l < e; ++l) {
+      int len = std::min(n_tok + 1, c->hs->layers[l].b);
+      int ns = (len + split - 1) / split;
+      any_split |= ns > 1;
+      n_items += (long long)U * ns;
+    }
+    if ((size_t)n_items > c->wl.items_cap) return fail(c, SQ_ERR_CAPACITY, "workspace too small for the split plan");
+    DecodeArgs a;
+    a.layers = ws_ptr<LayerDesc>(c, c->wl.layers);
+    a.order = ws_ptr<int>(c, c->wl.order);
+    a.pool = c->pool;
+    a.logits = ws_ptr<float>(c, c->wl.logits);
+    a.part_stat = ws_ptr<float>(c, c->wl.part_stat);
+    a.part_o = ws_ptr<float>(c, c->wl.part_o);
+    a.q = static_cast<const char*>(q) + (size_t)(s - layer_begin) * q_layer;
+    a.k_new = static_cast<const char*>(k_new) + (size_t)(s - layer_begin) * kv_layer;
+    a.v_new = static_cast<const char*>(v_new) + (size_t)(s - layer_begin) * kv_layer;
+    a.out = static_cast<char*>(out) + (size_t)(s - layer_begin) * q_layer;
+    a.status = ws_ptr<int>(c, c->wl.status);
+    a.n_layer_total = cfg.n_layer;
+    a.layer_begin = s;
+    a.layer_end = e;
+    a.n_tok = n_tok;
+    a.batch = c->batch;
+    a.n_q_head = cfg.n_q_head;
+    a.n_kv_head = cfg.n_kv_head;
+    a.head_dim = cfg.head_dim;
+    a.group = G;
+    a.n_unit = U;
+    a.split_tokens = split;
+    a.policy = cfg.policy;
+    a.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg.head_dim));
+    const bool combine = any_split || cfg.policy == SQ_POLICY_H2O;
+    SQ_CUDA(c, launch_decode(a, cfg.dtype, (int)n_items, combine, st));
+    for (int l = s; l < e; ++l) c->n_tok[l] += 1;
+    s = e;
+  }
+  return SQ_OK;
+}
+
+int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* new_budgets_host, void* stream) {
+  if (!c) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (layer_begin < 0 || layer_end > c->cfg.n_layer || layer_begin >= layer_end || !new_budgets_host)
+    return fail(c, SQ_ERR_INVALID_ARG, "layer range / budgets");
+  int rc = ensure_budgets(c, st);
+  if (rc != SQ_OK) return rc;
+  const sq_config& cfg = c->cfg;
+  for (int l = layer_begin; l < layer_end; ++l) {
+    const int nb = new_budgets_host[l - layer_begin];
+    if (!c->prefilled[l]) return fail(c, SQ_ERR_STATE, "sq_prefill_compress has not been called for a layer in the range");
+    if (nb < 1 || nb > c->hs->layers[l].b) return fail(c, SQ_ERR_INVALID_ARG, "new budget must be in 1..current budget");
+    if (cfg.policy == SQ_POLICY_STREAMING_LLM && nb <= cfg.n_sink)
+      return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
+  }
+  const int U = c->batch * cfg.n_kv_head;
+  for (int l = layer_begin; l < layer_end; ++l) {
+    const int nb = new_budgets_host[l - layer_begin];
+    LayerDesc old = c->hs->layers[l];
+    if (nb == old.b) continue;
+    LayerDesc nw = old;
+    nw.b = nb;
+    nw.b_heavy = cfg.policy == SQ_POLICY_H2O ? (int)(((long long)nb * cfg.heavy_num) / cfg.heavy_den) : 0;
+    nw.b_recent = nb - nw.b_heavy;
+    const int n_tok = c->n_tok[l];
+    const int len = std::min(n_tok, old.b);
+    if (cfg.policy != SQ_POLICY_H2O) {
+      // the compaction keeps slot order, so the ring stays a rotation: find its new phase
+      const int base = old.ring_base, r_old = old.b - base, r_new = nb - base;
+      if (n_tok <= nb) {
+        nw.ring_origin = base;
+      } else {
+        const int x0 = n_tok - r_new;
+        const int r0 = (x0 - old.ring_origin) % r_old;
+        const int h = (r0 + r_new <= r_old) ? 0 : r0 + r_new - r_old;
+        nw.ring_origin = x0 - h;
+      }
+    }
+    if (len > nb) {
+      EvictArgs a;
+      a.pool = c->pool;
+      a.ld_old = old;
+      a.ld_new = nw;
+      a.n_unit = U;
+      a.len = len;
+      a.n_tok = n_tok;
+      a.policy = cfg.policy;
+      a.n_sink = cfg.n_sink;
+      a.row_bytes = cfg.head_dim * elem_bytes(cfg.dtype);
+      a.status = ws_ptr<int>(c, c->wl.status);
+      SQ_CUDA(c, launch_evict(a, st));
+    }
+    c->hs->layers[l] = nw;
+    c->hs->budget[l] = nb;
+    rc = upload_layer(c, l, st);
+    if (rc != SQ_OK) return rc;
+  }
+  // the launch order (largest budget first) may have changed
+  std::vector<int> ord(cfg.n_layer);
+  for (int l = 0; l < cfg.n_layer; ++l) ord[l] = l;
+  std::stable_sort(ord.begin(), ord.end(), [&](int x, int y) { return c->hs->budget[x] > c->hs->budget[y]; });
+  std::copy(ord.begin(), ord.end(), c->hs->order);
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs->order, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs->budget, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaStreamSynchronize(st));
+  return SQ_OK;
+}
+
+int sq_get_cos_sim(sq_ctx* c, float* cos_sim_host) {
+  if (!c || !cos_sim_host) return SQ_ERR_INVALID_ARG;
+  if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "sq_allocate_budgets has not been called");
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  SQ_CUDA(c, cudaMemcpy(cos_sim_host, ws_ptr<float>(c, c->wl.cos_sim), 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  return SQ_OK;
+}
+
+int sq_get_budgets(sq_ctx* c, int32_t* budgets_host, uint8_t* is_g3_host) {
+  if (!c || !budgets_host) return SQ_ERR_INVALID_ARG;
+  if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "budgets not set");
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  SQ_CUDA(c, cudaMemcpy(budgets_host, ws_ptr<int>(c, c->wl.budget), 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  if (is_g3_host)
+    SQ_CUDA(c, cudaMemcpy(is_g3_host, ws_ptr<unsigned char>(c, c->wl.is_g3), c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  return SQ_OK;
+}
+
+static int unit_order(sq_ctx* c, int layer, int seq, int kv_head, std::vector<int>& pos, std::vector<int>& order) {
+  if (layer < 0 || layer >= c->cfg.n_layer || seq < 0 || seq >= c->batch || kv_head < 0 || kv_head >= c->cfg.n_kv_head)
+    return fail(c, SQ_ERR_INVALID_ARG, "layer/seq/kv_head out of range");
+  if (c->budget_state != 2 || !c->prefilled[layer]) return fail(c, SQ_ERR_STATE, "layer has no cache yet");
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  const LayerDesc& ld = c->hs->layers[layer];
+  const int len = std::min(c->n_tok[layer], ld.b);
+  const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
+  pos.resize(len);
+  SQ_CUDA(c, cudaMemcpy(pos.data(), c->pool + ld.pos_off + unit * ld.cap * 4, (size_t)len * 4, cudaMemcpyDeviceToHost));
+  order.resize(len);
+  for (int i = 0; i < len; ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](int x, int y) { return pos[x] < pos[y]; });
+  return SQ_OK;
+}
+
+int sq_get_kept(sq_ctx* c, int32_t layer, int32_t seq, int32_t kv_head, int32_t* pos_host, float* acc_host, int32_t* n) {
+  if (!c || !pos_host || !n) return SQ_ERR_INVALID_ARG;
+  std::vector<int> pos, order;
+  int rc = unit_order(c, layer, seq, kv_head, pos, order);
+  if (rc != SQ_OK) return rc;
+  const LayerDesc& ld = c->hs->layers[layer];
+  const int len = (int)pos.size();
+  std::vector<float> acc(len, 0.f);
+  if (c->cfg.policy == SQ_POLICY_H2O && len > 0) {
+    const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
+    SQ_CUDA(c, cudaMemcpy(acc.data(), c->pool + ld.acc_off + unit * ld.cap * 4, (size_t)len * 4, cudaMemcpyDeviceToHost));
+  }
+  for (int i = 0; i < len; ++i) {
+    pos_host[i] = pos[order[i]];
+    if (acc_host) acc_host[i] = acc[order[i]];
+  }
+  *n = len;
+  return SQ_OK;
+}
+
+int sq_get_kv(sq_ctx* c, int32_t layer, int32_t seq, int32_t kv_head, void* k_host, void* v_host) {
+  if (!c || !k_host || !v_host) return SQ_ERR_INVALID_ARG;
+  std::vector<int> pos, order;
+  int rc = unit_order(c, layer, seq, kv_head, pos, order);
+  if (rc != SQ_OK) return rc;
+  const LayerDesc& ld = c->hs->layers[layer];
+  const int len = (int)pos.size();
+  const size_t row = (size_t)c->cfg.head_dim * elem_bytes(c->cfg.dtype);
+  const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
+  std::vector<char> kb(len * row), vb(len * row);
+  if (len > 0) {
+    SQ_CUDA(c, cudaMemcpy(kb.data(), c->pool + ld.k_off + unit * ld.cap * row, len * row, cudaMemcpyDeviceToHost));
+    SQ_CUDA(c, cudaMemcpy(vb.data(), c->pool + ld.v_off + unit * ld.cap * row, len * row, cudaMemcpyDeviceToHost));
+  }
+  for (int i = 0; i < len; ++i) {
+    std::memcpy(static_cast<char*>(k_host) + i * row, kb.data() + order[i] * row, row);
+    std::memcpy(static_cast<char*>(v_host) + i * row, vb.data() + order[i] * row, row);
+  }
+  return SQ_OK;
+}
+
+int sq_get_len(sq_ctx* c, int32_t layer, int32_t* len) {
+  if (!c || !len) return SQ_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layer) return fail(c, SQ_ERR_INVALID_ARG, "layer out of range");
+  if (c->budget_state != 2 || !c->prefilled[layer]) return fail(c, SQ_ERR_STATE, "layer has no cache yet");
+  *len = std::min(c->n_tok[layer], c->hs->layers[layer].b);
+  return SQ_OK;
+}
+
+int sq_status(sq_ctx* c, int32_t* device_status) {
+  if (!c || !device_status) return SQ_ERR_INVALID_ARG;
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  SQ_CUDA(c, cudaMemcpy(device_status, ws_ptr<int>(c, c->wl.status), 4, cudaMemcpyDeviceToHost));
+  return SQ_OK;
+}
+
+int sq_kv_bytes_per_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, int64_t* bytes) {
+  if (!c || !bytes) return SQ_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end > c->cfg.n_layer || layer_begin >= layer_end)
+    return fail(c, SQ_ERR_INVALID_ARG, "layer range");
+  if (c->budget_state != 2) return fail(c, SQ_ERR_STATE, "budgets not on the host yet");
+  const int64_t U = (int64_t)c->batch * c->cfg.n_kv_head;
+  const int64_t row = (int64_t)c->cfg.head_dim * elem_bytes(c->cfg.dtype);
+  int64_t total = 0;
+  for (int l = layer_begin; l < layer_end; ++l)
+    total += U * std::min(c->n_tok[l] + 1, c->hs->layers[l].b) * 2 * row;
+  *bytes = total;
+  return SQ_OK;
+}
+
+}  // extern "C"
