@@ -335,7 +335,7 @@ def test_call_order_and_argument_errors():
         ctx.prefill_compress(0, k, v)            # no budgets yet
     assert e.value.code == B.SQ_ERR_STATE
     with pytest.raises(B.SqError) as e:
-        ctx.set_budgets([31, 31, 31])            # does not fit the pool sized for 3 * 30
+        ctx.set_budgets([60, 60, 60])            # does not fit the pool sized for 3 * 30
     assert e.value.code == B.SQ_ERR_CAPACITY
     ctx.set_budgets([30, 30, 30])
     dq, dk, dv = synth.decode_qkv(w, 0, DEV)
