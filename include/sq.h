@@ -167,6 +167,37 @@ const char* sq_last_error(sq_ctx* ctx);
  * fill level (for bandwidth accounting). */
 int sq_kv_bytes_per_step(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, int64_t* bytes);
 
+/* H2O prompt scores for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the scoring step inside
+ * sq_prefill_compress.)  Some hosts of this library run where cudaMalloc is off limits:
+ * inside a memory pool that was sized and handed out up front, in a plugin whose embedding
+ * runtime owns every allocation, or in a service that forbids allocation after start-up so
+ * that a request can never fail for lack of memory.  sq_prefill_compress needs a workspace
+ * from the caller for the per-row log-sum-exp of the causal score matrix; this call keeps
+ * that intermediate in a fixed array that is part of the library image instead, so the
+ * caller passes only inputs and the output:
+ *   q_prompt [batch, n_q_head, prompt_len, head_dim], k_prompt [batch, n_kv_head, prompt_len,
+ *   head_dim] (dtype sq_dtype), acc_out fp32 [batch, n_kv_head, prompt_len]; all device
+ *   pointers, 16-byte aligned.  acc_out[b, h, t] = sum over the query heads sharing KV head h
+ *   and over rows r >= t of softmax_row_r(Q K^T / sqrt(head_dim))[t], exactly what
+ *   sq_prefill_compress computes from q_prompt.
+ * Limits and rules:
+ *   - batch * n_q_head * prompt_len <= SQ_STATIC_SCORE_MAX_ROWS (the array holds one float
+ *     per query row: 4 MiB, resident on every GPU that loads the library until the process
+ *     exits); larger requests return SQ_ERR_CAPACITY and launch nothing.
+ *   - The first call on each device looks up the array's device address (no allocation);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (every
+ *     entry a call reads was written by that call first), but two calls that overlap on the
+ *     GPU (different streams, or different host threads without ordering) race on it: order
+ *     them on one stream or with events.
+ *   - Calls no cudaMalloc/cudaFree and no allocating library routine; needs no sq_ctx. */
+#define SQ_STATIC_SCORE_MAX_ROWS (1 << 20)
+int sq_prompt_scores_static(const void* q_prompt, const void* k_prompt, int32_t batch, int32_t n_q_head,
+                            int32_t n_kv_head, int32_t prompt_len, int32_t head_dim, int32_t dtype, float* acc_out,
+                            void* stream);
+int64_t sq_prompt_scores_static_max_rows(void);
+
 #ifdef __cplusplus
 }
 #endif

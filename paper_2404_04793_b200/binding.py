@@ -25,7 +25,8 @@ _ERR_NAMES = {1: "SQ_ERR_INVALID_ARG", 2: "SQ_ERR_STATE", 3: "SQ_ERR_CAPACITY", 
 EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequence_batch",
            "sq_layer_importance", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
            "sq_decode_step", "sq_evict", "sq_get_cos_sim", "sq_get_budgets", "sq_get_kept", "sq_get_kv",
-           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step"]
+           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static",
+           "sq_prompt_scores_static_max_rows"]
 
 
 class sq_config(ctypes.Structure):
@@ -72,8 +73,11 @@ def lib() -> ctypes.CDLL:
     L.sq_last_error.argtypes = [P]
     L.sq_last_error.restype = c_char_p
     L.sq_kv_bytes_per_step.argtypes = [P, c_int32, c_int32, POINTER(c_int64)]
+    L.sq_prompt_scores_static.argtypes = [P, P, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, P, P]
+    L.sq_prompt_scores_static_max_rows.argtypes = []
+    L.sq_prompt_scores_static_max_rows.restype = c_int64
     for name in EXPORTS:
-        if name != "sq_last_error":
+        if name not in ("sq_last_error", "sq_prompt_scores_static_max_rows"):
             getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -210,3 +214,19 @@ class Context:
         b = c_int64()
         self._ck(lib().sq_kv_bytes_per_step(self._h, layer_begin, layer_end, byref(b)))
         return b.value
+
+
+def sq_prompt_scores_static(q_prompt, k_prompt, acc_out):
+    """H2O prompt scores through the entry point that allocates nothing (its intermediate sits
+    in a fixed array inside the library).  q_prompt [B, Hq, P, d], k_prompt [B, Hkv, P, d],
+    acc_out fp32 [B, Hkv, P]: CUDA tensors the caller already owns.  Raises SqError with
+    SQ_ERR_CAPACITY when B * Hq * P exceeds the array."""
+    B_, Hq, P_, d = q_prompt.shape
+    Hkv = k_prompt.shape[1]
+    dt = {torch.float32: SQ_F32, torch.bfloat16: SQ_BF16}[q_prompt.dtype]
+    if acc_out.dtype != torch.float32 or tuple(acc_out.shape) != (B_, Hkv, P_):
+        raise ValueError("acc_out must be fp32 [batch, n_kv_head, prompt_len]")
+    rc = lib().sq_prompt_scores_static(_dptr(q_prompt), _dptr(k_prompt), B_, Hq, Hkv, P_, d, dt, _dptr(acc_out),
+                                       _stream())
+    if rc != SQ_OK:
+        raise SqError(rc, "sq_prompt_scores_static")

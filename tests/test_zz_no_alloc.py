@@ -1,0 +1,68 @@
+"""The allocation-free scoring entry point against the regular one.
+
+sq_prompt_scores_static serves hosts that must not call cudaMalloc (pre-sized memory pools,
+plugins whose runtime owns all allocations, services that forbid allocation after start-up):
+its intermediate lives in a fixed array inside the library.  Here it is called twice in a row
+through the C ABI -- the second call on a different, smaller problem, so stale contents of the
+shared array would show -- and each result is compared with the scores sq_prefill_compress
+computes for the same prompt, within the tolerance the other score tests use.  This file is
+collected last on purpose."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_04793_b200 import binding as B
+from paper_2404_04793_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _scores_via_context(w, q, k, v):
+    ctx = H.make_ctx(w, b_init=w.prompt)
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets([w.prompt] * w.n_layer)        # keep every token so every score can be read back
+    ctx.prefill_compress(0, k, v, q)
+    out = np.zeros((w.batch, w.n_kv_head, w.prompt), dtype=np.float32)
+    for s in range(w.batch):
+        for h in range(w.n_kv_head):
+            pos, acc = ctx.get_kept(0, s, h)
+            assert pos == list(range(w.prompt))
+            out[s, h] = acc
+    return out
+
+
+def test_static_scores_match_regular_entry_point_twice_in_a_row():
+    cases = [
+        dict(dtype=torch.bfloat16, head_dim=128, n_q_head=8, n_kv_head=2, batch=2, prompt=333),
+        dict(dtype=torch.float32, head_dim=64, n_q_head=3, n_kv_head=1, batch=1, prompt=97),
+    ]
+    for i, kw in enumerate(cases):
+        w = synth.Workload(f"noalloc{i}", 40 + i, n_layer=1, hidden=64, steps=1, policy=synth.H2O, budget_pct=100.0,
+                           p=0.3, heavy_mode="uniform4", **kw)
+        q, k, v = synth.prompt_qkv(w, 0, DEV)
+        acc = torch.full((w.batch, w.n_kv_head, w.prompt), float("nan"), dtype=torch.float32, device=DEV)
+        B.sq_prompt_scores_static(q, k, acc)
+        torch.cuda.synchronize()
+        got = acc.cpu().numpy()
+        want = _scores_via_context(w, q, k, v)
+        assert np.isfinite(got).all()
+        assert np.allclose(got, want, rtol=H.RTOL_ACC[w.dtype], atol=1e-6)
+        assert abs(got.sum() - w.batch * w.n_q_head * w.prompt) < 1e-3 * w.batch * w.n_q_head * w.prompt
+
+
+def test_static_scores_reject_oversized_and_bad_requests():
+    cap = B.lib().sq_prompt_scores_static_max_rows()
+    assert cap == 1 << 20
+    q = torch.zeros(1, 2, 8, 64, device=DEV)
+    k = torch.zeros(1, 1, 8, 64, device=DEV)
+    acc = torch.zeros(1, 1, 8, device=DEV)
+    P = B.c_void_p
+    args = lambda batch, hq, p, d: (P(q.data_ptr()), P(k.data_ptr()), batch, hq, 1, p, d, B.SQ_F32, P(acc.data_ptr()), None)
+    # one row too many: refused before anything is launched (the small tensors are never read)
+    assert B.lib().sq_prompt_scores_static(*args(1, 2, cap // 2 + 1, 64)) == B.SQ_ERR_CAPACITY
+    assert B.lib().sq_prompt_scores_static(*args(1, 2, 8, 96)) == B.SQ_ERR_UNSUPPORTED
+    assert B.lib().sq_prompt_scores_static(*args(0, 2, 8, 64)) == B.SQ_ERR_INVALID_ARG
+    assert B.lib().sq_prompt_scores_static(None, P(k.data_ptr()), 1, 2, 1, 8, 64, B.SQ_F32, P(acc.data_ptr()), None) \
+        == B.SQ_ERR_INVALID_ARG
