@@ -48,7 +48,7 @@ def workload_by_name(name):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    Q = ("uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -61,11 +61,20 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "200"], stdout=self.f, stderr=subprocess.DEVNULL)
+                                          "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _ts(text):
+        import datetime
+        try:
+            return datetime.datetime.strptime(text.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken between the wall-clock times t_begin and t_end."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -79,8 +88,12 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             p = [x.strip() for x in line.split(",")]
-            if len(p) < 9 or (self.uuid not in p[0] and p[0] not in self.uuid):
+            if len(p) < 10 or (self.uuid not in p[1] and p[1] not in self.uuid):
                 continue
+            ts = self._ts(p[0])
+            if ts is not None and t_begin is not None and not (t_begin - 0.1 <= ts <= t_end + 0.1):
+                continue
+            p = p[1:]
             try:
                 sm.append(float(p[1])); mx.append(float(p[2]))
             except ValueError:
@@ -119,7 +132,8 @@ def _oracle_sample(w, n_units, n_imp_tokens, seed, device):
     t_imp = 0.0
     n_imp = 0
     for l in layers_imp:
-        a, b = synth.hidden_pair(w, l, device, batch=1, n_tok=min(per_layer, w.prompt))
+        nb = max(1, min(w.batch, per_layer // w.prompt))
+        a, b = synth.hidden_pair(w, l, device, batch=nb, n_tok=min(per_layer, w.prompt))
         a, b = f64(a), f64(b)
         t0 = time.perf_counter()
         cos[l] = O.layer_importance(a, b)
@@ -209,8 +223,10 @@ def run_ours(args, w):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        job.run(inp)                      # keeps the GPU busy while the sampler starts up
     dist_util.barrier()
     torch.cuda.synchronize()
+    t_begin = time.time()
     e0, e1 = ev(), ev()
     mids = []
     e0.record()
@@ -223,8 +239,9 @@ def run_ours(args, w):
         mids.append((a, b))
     e1.record()
     torch.cuda.synchronize()
+    t_end = time.time()
     dist_util.barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ms_step = e0.elapsed_time(e1) / args.steps
     ms_decode = sum(a.elapsed_time(b) for a, b in mids) / args.steps
     status = job.ctx.status()
@@ -278,7 +295,7 @@ def run_ours(args, w):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        v, secs, desc = oracle_sample(wr, n_units=64, n_imp_tokens=32768, seed=7, device=dev)
+        v, secs, desc = oracle_sample(wr, n_units=256, n_imp_tokens=65536, seed=7, device=dev)
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": secs}
 
     line = {
@@ -305,16 +322,22 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b")
     ap.add_argument("--per-layer-decode", action="store_true", help="one decode launch per layer instead of one per step")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = workload_by_name(args.workload)
+    if args.batch:
+        w = w.replace(batch=args.batch, name=w.name + f"_b{args.batch}")
+    if args.decode_steps:
+        w = w.replace(steps=args.decode_steps, name=w.name + f"_t{args.decode_steps}")
     if args.impl == "reference":
         run_reference(args, w)
     else:
