@@ -2,61 +2,15 @@
 // token into the slot C_seq frees, attend over the kept slots (split-K flash-decode, all query
 // heads of a KV head share one pass over K/V), and for H2O add the received probabilities to
 // the per-token scores and choose the slot the next append will reuse.
+#include <cstdlib>
+#include <cstring>
+
 #include "sq_device.cuh"
 #include "sq_internal.h"
 #include "sq_select.cuh"
+#include "sq_decode_common.cuh"
 
 namespace sq {
-
-constexpr unsigned kFull = 0xffffffffu;
-
-struct ItemLoc {
-  int layer, local, n_split, base;
-};
-
-__device__ __forceinline__ int n_split_of(const DecodeArgs& a, int b) {
-  int len = min(a.n_tok + 1, b);
-  return (len + a.split_tokens - 1) / a.split_tokens;
-}
-
-// Work items of a launch are numbered layer by layer in `order` (largest budget first), and
-// within a layer as unit * n_split + split.  Each warp finds, by a prefix scan over the
-// layers, either the layer an item index falls in (want_layer < 0) or the first item of a
-// given layer.
-__device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_layer, ItemLoc& out) {
-  const int lane = threadIdx.x & 31;
-  int running = 0;
-  for (int c = 0; c < a.n_layer_total; c += 32) {
-    const int i = c + lane;
-    int l = -1, ns = 0, cnt = 0;
-    if (i < a.n_layer_total) {
-      int li = a.order[i];
-      if (li >= a.layer_begin && li < a.layer_end) {
-        l = li;
-        ns = n_split_of(a, a.layers[li].b);
-        cnt = a.n_unit * ns;
-      }
-    }
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int t = __shfl_up_sync(kFull, incl, o);
-      if (lane >= o) incl += t;
-    }
-    unsigned hit = (want_layer >= 0) ? __ballot_sync(kFull, l == want_layer)
-                                     : __ballot_sync(kFull, cnt > 0 && idx < running + incl);
-    if (hit) {
-      const int src = __ffs(hit) - 1;
-      out.layer = __shfl_sync(kFull, l, src);
-      out.n_split = __shfl_sync(kFull, ns, src);
-      out.base = running + __shfl_sync(kFull, incl - cnt, src);
-      out.local = idx - out.base;
-      return true;
-    }
-    running += __shfl_sync(kFull, incl, 31);
-  }
-  return false;
-}
 
 // One CTA (4 warps) per (layer, unit, split).  A K or V row is D*sizeof(T) bytes = LPR lanes
 // x 16 bytes, so a warp reads 32/LPR consecutive rows per load instruction, fully coalesced.
@@ -101,7 +55,7 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
   const T* vn = reinterpret_cast<const T*>(a.v_new) + (tok * a.n_kv_head + kvh) * D;
   T* ob = reinterpret_cast<T*>(a.out) + (tok * a.n_q_head + (size_t)kvh * a.group) * D;
   float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * a.group;  // [slot][group]
-  float* stat = a.part_stat + (size_t)blockIdx.x * a.group * 2;
+  float* stat = a.part_stat + (size_t)blockIdx.x * a.group * kStatStride;
   float* po = a.part_o + (size_t)blockIdx.x * a.group * D;
 
   for (int hb = 0; hb < a.group; hb += GT) {
@@ -238,8 +192,9 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
       else
         po[(size_t)h * D + e] = O;
       if (e == 0) {
-        stat[h * 2] = M;
-        stat[h * 2 + 1] = L;
+        stat[h * kStatStride] = M;
+        stat[h * kStatStride + 1] = L;
+        stat[h * kStatStride + 2] = L;
       }
     }
     __syncthreads();
@@ -267,7 +222,7 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
 template <typename T>
 __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
   __shared__ SelScratch sc;
-  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup];
+  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
   const int n_layers = a.layer_end - a.layer_begin;
   const int layer = a.layer_begin + blockIdx.x / a.n_unit;
   const int unit = blockIdx.x % a.n_unit;
@@ -278,17 +233,20 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
   const LayerDesc* ldp = a.layers + layer;
   const int b = ldp->b, cap = ldp->cap;
   const size_t item0 = (size_t)it.base + (size_t)unit * ns;
-  const float* stat = a.part_stat + item0 * G * 2;
+  const float* stat = a.part_stat + item0 * G * kStatStride;
   for (int h = tid; h < G; h += kSelThreads) {
     float M = -INFINITY;
-    for (int s = 0; s < ns; ++s) M = fmaxf(M, stat[((size_t)s * G + h) * 2]);
-    float L = 0.f;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, stat[((size_t)s * G + h) * kStatStride]);
+    float L = 0.f, Lw = 0.f;
     for (int s = 0; s < ns; ++s) {
-      const float ms = stat[((size_t)s * G + h) * 2];
-      L += stat[((size_t)s * G + h) * 2 + 1] * ((ms > -INFINITY) ? exp2f(ms - M) : 0.f);
+      const float* st = stat + ((size_t)s * G + h) * kStatStride;
+      const float f = (st[0] > -INFINITY) ? exp2f(st[0] - M) : 0.f;
+      L += st[1] * f;
+      Lw += st[2] * f;
     }
     s_M[h] = M;
-    s_invL[h] = 1.f / L;
+    s_invL[h] = 1.f / L;     // normaliser of the probabilities (H2O scores)
+    s_invLw[h] = 1.f / Lw;   // normaliser matching the weights the output was accumulated with
   }
   __syncthreads();
   if (ns > 1) {
@@ -300,10 +258,10 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
       const int h = idx / D;
       float O = 0.f;
       for (int s = 0; s < ns; ++s) {
-        const float ms = stat[((size_t)s * G + h) * 2];
+        const float ms = stat[((size_t)s * G + h) * kStatStride];
         O += po[(size_t)s * G * D + idx] * ((ms > -INFINITY) ? exp2f(ms - s_M[h]) : 0.f);
       }
-      ob[idx] = narrow<T>(O * s_invL[h]);
+      ob[idx] = narrow<T>(O * s_invLw[h]);
     }
   }
   if (a.policy != SQ_POLICY_H2O) return;
@@ -347,9 +305,29 @@ static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
     decode_attn_kernel<T, D, 8><<<n_items, 128, 0, s>>>(a);
 }
 
+// Which attention kernel serves a shape: grouped bf16 heads go to the tensor-core kernel,
+// everything else (fp32, one query head per KV head, shapes it does not cover) to the fp32-pipe
+// kernel.  SQ_DECODE_PATH=alu|mma overrides the choice (for A/B measurements).
+static int decode_path_override() {
+  static int mode = -1;
+  if (mode < 0) {
+    const char* e = getenv("SQ_DECODE_PATH");
+    mode = !e ? 0 : (!strcmp(e, "alu") ? 1 : (!strcmp(e, "mma") ? 2 : 0));
+  }
+  return mode;
+}
+
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, cudaStream_t s) {
   if (n_items <= 0) return cudaSuccess;
-  if (dtype == SQ_F32) {
+  const int ovr = decode_path_override();
+  bool done = false;
+  if (dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
+    cudaError_t e = launch_decode_attn_mma(a, n_items, s);
+    if (e == cudaSuccess) done = true;
+    else if (e != cudaErrorNotSupported) return e;
+  }
+  if (done) {
+  } else if (dtype == SQ_F32) {
     if (a.head_dim == 64) launch_attn_g<float, 64>(a, n_items, s);
     else launch_attn_g<float, 128>(a, n_items, s);
   } else {

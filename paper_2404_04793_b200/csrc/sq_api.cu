@@ -116,7 +116,7 @@ WsLayout ws_layout(const sq_config& c, int64_t b_init) {
   w.layers = take(sizeof(LayerDesc) * L);
   w.order = take(4 * L);
   w.items_cap = (size_t)kTargetItems + U * L;
-  w.part_stat = take(w.items_cap * G * 2 * 4);
+  w.part_stat = take(w.items_cap * G * 4 * 4);
   w.part_o = take(w.items_cap * G * c.head_dim * 4);
   const bool h2o = c.policy == SQ_POLICY_H2O;
   w.logits_floats = h2o ? U * G * (L * (size_t)b_init + L * (c.page_tokens - 1)) : 0;

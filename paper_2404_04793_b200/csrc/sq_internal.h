@@ -74,7 +74,7 @@ struct DecodeArgs {
   const int* order;  // layer indices sorted by budget, descending
   char* pool;
   float* logits;
-  float* part_stat;  // [item][group][2]   (max, sum) in the log2 domain
+  float* part_stat;  // [item][group][4]   (max, sum, sum of rounded weights, pad) in the log2 domain
   float* part_o;     // [item][group][head_dim]
   const void* q;
   const void* k_new;
@@ -105,6 +105,7 @@ cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt
                                  cudaStream_t s);
 cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int len, int next_pos, cudaStream_t s);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, cudaStream_t s);
+cudaError_t launch_decode_attn_mma(const DecodeArgs& a, int n_items, cudaStream_t s);
 cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s);
 
 }  // namespace sq

@@ -223,7 +223,8 @@ def test_tiny_config_full_trajectory():
 @pytest.mark.parametrize("dtype,head_dim,hq,hkv", [
     (torch.float32, 64, 2, 2), (torch.float32, 128, 8, 2), (torch.bfloat16, 128, 4, 4),
     (torch.bfloat16, 128, 8, 2), (torch.bfloat16, 128, 16, 2), (torch.bfloat16, 64, 71, 1),
-    (torch.bfloat16, 64, 6, 2)])
+    (torch.bfloat16, 64, 6, 2), (torch.bfloat16, 128, 20, 1), (torch.bfloat16, 64, 48, 2),
+    (torch.bfloat16, 128, 40, 1)])
 def test_decode_small_shapes(policy, dtype, head_dim, hq, hkv):
     w = small("dec", 19, policy=policy, dtype=dtype, head_dim=head_dim, n_q_head=hq, n_kv_head=hkv,
               heavy_mode="uniform4", steps=7)
