@@ -35,9 +35,9 @@ from paper_2404_04793_b200 import dist_util, synth
 METRIC = "decode tokens/sec at 1 B200 and fused attn+evict HBM GB/s as % of roofline"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram bytes (read+write) per decode launch from the ncu capture summarised under profiles/;
-# None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram bytes (read+write) per decode launch of the default workload, from the ncu capture
+# summarised in profiles/decode_attn_llama2_7b_sw_b2.md (batch-2 capture scaled by 4 to batch 8).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama2_7b_sw_bf16": 1.7364e9}
 
 
 def workload_by_name(name):
@@ -289,7 +289,7 @@ def run_ours(args, w):
     else:
         peak = FALLBACK_HBM_GBS; peak_kind = "fallback"
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": peak_kind, "kernel": "decode_attn_kernel",
+                "traffic": None if args.per_layer_decode else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wr.name), "peak_kind": peak_kind, "kernel": "decode_attn_kernel",
                 "algorithmic_bytes_per_launch": bytes_per_launch, "us_per_launch": sec_per_launch * 1e6,
                 "frac_of_nominal_8000": achieved / 8000.0}
 
