@@ -1,6 +1,9 @@
 // Prefill side of Algorithm 1 (step 13 with the first compression of steps 16-18 applied at
 // once): H2O prompt scores, C_seq selection over the prompt, and the gather of the kept K/V
 // rows into the layer's cache region.
+#include <cstdlib>
+#include <cstring>
+
 #include "sq_device.cuh"
 #include "sq_internal.h"
 #include "sq_select.cuh"
@@ -156,11 +159,27 @@ static cudaError_t launch_scores_t(const ScoreArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, cudaStream_t s) {
+// fp32-pipe kernels (any dtype)
+cudaError_t launch_prefill_scores_alu(const ScoreArgs& a, int dtype, cudaStream_t s) {
   if (dtype == SQ_F32) {
     return a.head_dim == 64 ? launch_scores_t<float, 64>(a, s) : launch_scores_t<float, 128>(a, s);
   }
   return a.head_dim == 64 ? launch_scores_t<__nv_bfloat16, 64>(a, s) : launch_scores_t<__nv_bfloat16, 128>(a, s);
+}
+
+// bf16 prompts go to the tcgen05 kernels; fp32 (and anything those cannot serve) stays on the
+// fp32 pipes.  SQ_PREFILL_PATH=alu forces the latter (for A/B measurements).
+cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, int* status, cudaStream_t s) {
+  static int force_alu = -1;
+  if (force_alu < 0) {
+    const char* e = getenv("SQ_PREFILL_PATH");
+    force_alu = (e && !strcmp(e, "alu")) ? 1 : 0;
+  }
+  if (dtype == SQ_BF16 && !force_alu) {
+    cudaError_t e = launch_prefill_scores_tc(a, status, s);
+    if (e != cudaErrorNotSupported) return e;
+  }
+  return launch_prefill_scores_alu(a, dtype, s);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -1,0 +1,381 @@
+// H2O prompt scores on the 5th-generation tensor cores (bf16).
+//
+// acc[t] = sum over the query heads sharing a KV head and over query rows r >= t of
+//          softmax_row_r(Q K^T / sqrt(d))[t]                       (causal)
+// is two sweeps over 128x128 tiles of the score matrix, each tile one tcgen05.mma chain
+// (M = N = 128, K = head_dim, bf16 in, fp32 accumulators in tensor memory):
+//   sweep 1, CTA = (sequence, query head, 128 query rows): S = Q_tile K_tile^T for the key tiles
+//     up to the diagonal; thread r of the four softmax warps owns TMEM lane r = one query row and
+//     keeps its running max / sum -> row log-sum-exp.
+//   sweep 2, CTA = (sequence, KV head, 128 keys): the operands swap, S^T = K_tile Q_tile^T for all
+//     query tiles from the diagonal down and all heads of the group; thread t owns one key and
+//     adds exp2(s*scale - lse[row]) over the tile's columns -> the key's column sum, with no
+//     cross-thread reduction and no atomics (deterministic).
+// Roles per CTA (6 warps): warp 0 issues TMA tile loads (128-byte swizzle, no multicast) into
+// a ring of shared-memory stages; warp 1 allocates tensor memory and issues the MMAs, signalling
+// completion through tcgen05.commit -> mbarrier; warps 2-5 drain the accumulators with
+// tcgen05.ld.  Two accumulator buffers let the next tile's MMA run under this tile's exponentials.
+// Every mbarrier wait is bounded: on expiry the CTA raises a status bit and winds down.
+#include <cuda.h>
+
+#include "sq_internal.h"
+
+namespace sq {
+
+namespace {
+
+constexpr int kTM = 128;                 // tile rows (TMEM lanes) and columns
+constexpr int kSubBytes = kTM * 128;     // one [128 rows x 64 bf16] swizzled sub-tile
+constexpr int kSpinLimit = 1 << 22;
+constexpr int kStatusTimeout = 16;
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for the phase with the given parity, giving up after kSpinLimit polls or once another
+// role has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255) == 255 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<unsigned long long>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+// shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ unsigned long long umma_desc(uint32_t saddr) {
+  return (unsigned long long)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+}  // namespace
+
+// SWEEP 1: rows = queries, streamed tiles = keys; SWEEP 2: rows = keys, streamed tiles = queries.
+template <int D, int STAGES, int SWEEP>
+__global__ void __launch_bounds__(192, 1)
+    prefill_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_rows, const __grid_constant__ CUtensorMap tm_stream,
+                             ScoreArgs a, float scale_log2, int* status) {
+  constexpr int SUB = D / 64;                  // 64-column sub-tiles per operand tile
+  constexpr int TILE_BYTES = SUB * kSubBytes;  // one operand tile
+  constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTM >> 3) << 17) | ((uint32_t)(kTM >> 4) << 24);
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* a_s = smem;
+  unsigned char* b_s = smem + TILE_BYTES;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(b_s + STAGES * TILE_BYTES);
+  // barriers (at most 15 of the 16 slots), then the TMEM base, the abort flag and the lse staging
+  static_assert(7 + 2 * STAGES <= 16, "barrier block");
+  const uint32_t bar_a = s_u32(bars + 0);
+  auto bar_full = [&](int s) { return s_u32(bars + 1 + s); };
+  auto bar_empty = [&](int s) { return s_u32(bars + 1 + STAGES + s); };
+  auto bar_sfull = [&](int b) { return s_u32(bars + 1 + 2 * STAGES + b); };
+  auto bar_sfree = [&](int b) { return s_u32(bars + 3 + 2 * STAGES + b); };
+  auto bar_lse = [&](int b) { return s_u32(bars + 5 + 2 * STAGES + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* lse_s = reinterpret_cast<float*>(tmem_slot + 4);  // [2][128], sweep 2 only
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int P = a.prompt, g = a.n_q_head / a.n_kv_head;
+  const int n_tile = (P + kTM - 1) / kTM;
+  const int bi = blockIdx.z;
+  int row_tile, n_stream;
+  long long rows0;  // first row of this CTA's fixed tile in the rows tensor
+  int hq = 0, hk = 0;
+  if (SWEEP == 1) {
+    hq = blockIdx.y;
+    hk = hq / g;
+    row_tile = n_tile - 1 - blockIdx.x;  // longest rows first
+    n_stream = row_tile + 1;
+    rows0 = ((long long)bi * a.n_q_head + hq) * P + (long long)row_tile * kTM;
+  } else {
+    hk = blockIdx.y;
+    row_tile = blockIdx.x;               // key tile 0 sees every query tile: longest first
+    n_stream = g * (n_tile - row_tile);
+    rows0 = ((long long)bi * a.n_kv_head + hk) * P + (long long)row_tile * kTM;
+  }
+  // first row of streamed tile i, and (sweep 2) its head / query tile
+  auto stream_row0 = [&](int i, int& h_out, int& qt_out) -> long long {
+    if (SWEEP == 1) {
+      h_out = 0;
+      qt_out = i;
+      return ((long long)bi * a.n_kv_head + hk) * P + (long long)i * kTM;
+    }
+    const int per = n_tile - row_tile;
+    h_out = i / per;
+    qt_out = row_tile + (i - h_out * per);
+    return ((long long)bi * a.n_q_head + hk * g + h_out) * P + (long long)qt_out * kTM;
+  };
+
+  if (tid == 0) {
+    mbar_init(bar_a, 1);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full(s), 1);
+      mbar_init(bar_empty(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_sfull(b), 1);
+      mbar_init(bar_sfree(b), 128);
+      mbar_init(bar_lse(b), 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(s_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      mbar_expect_tx(bar_a, TILE_BYTES);
+#pragma unroll
+      for (int sb = 0; sb < SUB; ++sb) tma_load_2d(s_u32(a_s + sb * kSubBytes), &tm_rows, sb * 64, (int)rows0, bar_a);
+      int issued = 0;
+      for (int i = 0; i < n_stream; ++i) {
+        const int st = i % STAGES;
+        if (i >= STAGES && !mbar_wait(bar_empty(st), ((i / STAGES) - 1) & 1, abort_flag)) break;
+        int h, qt;
+        const long long r0 = stream_row0(i, h, qt);
+        mbar_expect_tx(bar_full(st), TILE_BYTES);
+#pragma unroll
+        for (int sb = 0; sb < SUB; ++sb)
+          tma_load_2d(s_u32(b_s + st * TILE_BYTES + sb * kSubBytes), &tm_stream, sb * 64, (int)r0, bar_full(st));
+        issued = i + 1;
+      }
+      if (*abort_flag) {
+        // winding down early: let the copies already in flight land before the CTA exits
+        mbar_wait(bar_a, 0, abort_flag);
+        for (int i = max(0, issued - STAGES); i < issued; ++i) {
+          for (int k = 0; k < kSpinLimit && !mbar_try_wait(bar_full(i % STAGES), (i / STAGES) & 1); ++k) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    bool ok = mbar_wait(bar_a, 0, abort_flag);
+    for (int i = 0; ok && i < n_stream; ++i) {
+      const int st = i % STAGES, buf = i & 1;
+      ok = mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag);
+      if (ok && i >= 2) ok = mbar_wait(bar_sfree(buf), ((i >> 1) - 1) & 1, abort_flag);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (lane == 0) {
+        const uint32_t d_tmem = tmem_base + buf * kTM;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t a_addr = s_u32(a_s + (k / 4) * kSubBytes) + (k % 4) * 32;
+          const uint32_t b_addr = s_u32(b_s + st * TILE_BYTES + (k / 4) * kSubBytes) + (k % 4) * 32;
+          umma_bf16(d_tmem, umma_desc(a_addr), umma_desc(b_addr), kIdesc, k > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_empty(st));  // the stage may be refilled once these MMAs have read it
+        umma_commit(bar_sfull(buf)); // the accumulator buffer is complete
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------- accumulator drain: thread = one row of the fixed tile ----------------
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int row_idx = row_tile * kTM + row;  // query index (sweep 1) / key index (sweep 2)
+    const int t128 = (warp - 2) * 32 + lane;
+    float m = -INFINITY, l = 0.f, colsum = 0.f;
+    bool ok = true;
+    for (int i = 0; ok && i < n_stream; ++i) {
+      const int buf = i & 1;
+      int h, qt;
+      stream_row0(i, h, qt);
+      if (SWEEP == 2) {
+        const int q = qt * kTM + t128;
+        lse_s[buf * kTM + t128] = (q < P) ? a.lse2[((size_t)bi * a.n_q_head + hk * g + h) * P + q] : INFINITY;
+        mbar_arrive(bar_lse(buf));  // all 128 row sums of this query tile are staged
+        ok = mbar_wait(bar_lse(buf), (i >> 1) & 1, abort_flag);
+      }
+      if (ok) ok = mbar_wait(bar_sfull(buf), (i >> 1) & 1, abort_flag);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const bool diag = (qt == row_tile);
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTM + c * 32, v);
+        if (SWEEP == 1) {
+          if (diag) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j > row) v[j] = -INFINITY;  // key after the query
+          }
+          float mx = v[0];
+#pragma unroll
+          for (int j = 1; j < 32; ++j) mx = fmaxf(mx, v[j]);
+          const float m_new = fmaxf(m, mx * scale_log2);
+          if (m_new > -INFINITY) {
+            float sum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sum += ex2(fmaf(v[j], scale_log2, -m_new));
+            l = l * ex2(m - m_new) + sum;
+            m = m_new;
+          }
+        } else {
+          const float4* ls = reinterpret_cast<const float4*>(lse_s + buf * kTM + c * 32);
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) {
+            const float4 lv = ls[j4];
+            const float e0 = ex2(fmaf(v[4 * j4 + 0], scale_log2, -lv.x));
+            const float e1 = ex2(fmaf(v[4 * j4 + 1], scale_log2, -lv.y));
+            const float e2 = ex2(fmaf(v[4 * j4 + 2], scale_log2, -lv.z));
+            const float e3 = ex2(fmaf(v[4 * j4 + 3], scale_log2, -lv.w));
+            if (diag) {
+              const int q0 = c * 32 + 4 * j4;  // query before the key: no attention
+              colsum += (q0 + 0 >= row ? e0 : 0.f) + (q0 + 1 >= row ? e1 : 0.f) + (q0 + 2 >= row ? e2 : 0.f) +
+                        (q0 + 3 >= row ? e3 : 0.f);
+            } else {
+              colsum += (e0 + e1) + (e2 + e3);
+            }
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(bar_sfree(buf));
+    }
+    if (ok && row_idx < P) {
+      if (SWEEP == 1)
+        a.lse2[((size_t)bi * a.n_q_head + hq) * P + row_idx] = m + log2f(l);
+      else
+        a.acc_prompt[((size_t)bi * a.n_kv_head + hk) * P + row_idx] = colsum;
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
+  }
+  if (tid == 0 && *abort_flag) atomicOr(status, kStatusTimeout);
+}
+
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, d] bf16 row-major tensor, box = 128 rows x 64 columns, 128-byte swizzle
+static bool make_map(CUtensorMap* tm, const void* base, long long rows, int d) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)kTM};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int STAGES>
+static cudaError_t launch_tc_t(const ScoreArgs& a, int* status, cudaStream_t s) {
+  CUtensorMap tm_q, tm_k;
+  const long long q_rows = (long long)a.batch * a.n_q_head * a.prompt, k_rows = (long long)a.batch * a.n_kv_head * a.prompt;
+  if (q_rows + kTM > 0x7fffffffLL) return cudaErrorNotSupported;  // TMA coordinates are 32-bit
+  if (!make_map(&tm_q, a.q, q_rows, D) || !make_map(&tm_k, a.k, k_rows, D)) return cudaErrorNotSupported;
+  constexpr size_t smem = 1024 + (size_t)(1 + STAGES) * (D / 64) * kSubBytes + 8 * 16 + 16 + 2 * kTM * 4;
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  const int n_tile = (a.prompt + kTM - 1) / kTM;
+  auto k1 = prefill_scores_tc_kernel<D, STAGES, 1>;
+  auto k2 = prefill_scores_tc_kernel<D, STAGES, 2>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  k1<<<dim3(n_tile, a.n_q_head, a.batch), 192, smem, s>>>(tm_q, tm_k, a, scale_log2, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k2<<<dim3(n_tile, a.n_kv_head, a.batch), 192, smem, s>>>(tm_k, tm_q, a, scale_log2, status);
+  return cudaGetLastError();
+}
+
+// Returns cudaErrorNotSupported when the shape or the driver cannot serve the tensor-core path.
+cudaError_t launch_prefill_scores_tc(const ScoreArgs& a, int* status, cudaStream_t s) {
+  if (a.n_q_head > 65535 || a.batch > 65535) return cudaErrorNotSupported;
+  if ((reinterpret_cast<uintptr_t>(a.q) | reinterpret_cast<uintptr_t>(a.k)) & 15u) return cudaErrorNotSupported;
+  if (a.head_dim == 64) return launch_tc_t<64, 4>(a, status, s);
+  if (a.head_dim == 128) return launch_tc_t<128, 2>(a, status, s);
+  return cudaErrorNotSupported;
+}
+
+}  // namespace sq

@@ -387,7 +387,7 @@ int sq_prefill_compress(sq_ctx* c, int32_t layer, const void* k_prompt, const vo
       s.n_kv_head = c->cfg.n_kv_head;
       s.prompt = P;
       s.head_dim = c->cfg.head_dim;
-      SQ_CUDA(c, launch_prefill_scores(s, c->cfg.dtype, st));
+      SQ_CUDA(c, launch_prefill_scores(s, c->cfg.dtype, ws_ptr<int>(c, c->wl.status), st));
       acc = s.acc_prompt;
     }
     SQ_CUDA(c, launch_select_prompt(acc, U, P, ld, c->pool, st));

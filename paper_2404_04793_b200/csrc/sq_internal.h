@@ -100,7 +100,9 @@ struct EvictArgs {
 cudaError_t launch_importance(const ImportanceArgs& a, int dtype, int n_cta, cudaStream_t s);
 cudaError_t launch_allocate(const AllocateArgs& a, cudaStream_t s);
 cudaError_t launch_gather(const GatherArgs& a, int dtype, cudaStream_t s);
-cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, cudaStream_t s);
+cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, int* status, cudaStream_t s);
+cudaError_t launch_prefill_scores_alu(const ScoreArgs& a, int dtype, cudaStream_t s);
+cudaError_t launch_prefill_scores_tc(const ScoreArgs& a, int* status, cudaStream_t s);
 cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc& ld, char* pool,
                                  cudaStream_t s);
 cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int len, int next_pos, cudaStream_t s);

@@ -53,7 +53,7 @@ extern "C" int sq_prompt_scores_static(const void* q_prompt, const void* k_promp
   a.n_kv_head = n_kv_head;
   a.prompt = prompt_len;
   a.head_dim = head_dim;
-  if (sq::launch_prefill_scores(a, dtype, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SQ_ERR_CUDA;
+  if (sq::launch_prefill_scores_alu(a, dtype, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SQ_ERR_CUDA;
   return SQ_OK;
 }
 

@@ -120,9 +120,11 @@ def test_prefill_compress_keeps_what_cseq_keeps(policy, dtype, head_dim, budgets
 
 
 def test_h2o_prompt_scores_match_oracle():
-    for dtype, d, g in [(torch.float32, 64, 1), (torch.bfloat16, 128, 4), (torch.bfloat16, 64, 3)]:
+    for dtype, d, g, P in [(torch.float32, 64, 1, 150), (torch.bfloat16, 128, 4, 150), (torch.bfloat16, 64, 3, 150),
+                           (torch.bfloat16, 128, 2, 700), (torch.bfloat16, 64, 5, 513), (torch.bfloat16, 128, 1, 128),
+                           (torch.float32, 128, 2, 200)]:
         w = small("score", 16, policy=synth.H2O, dtype=dtype, head_dim=d, n_q_head=2 * g, n_kv_head=2,
-                  prompt=150, n_layer=1, heavy_mode="uniform4")
+                  prompt=P, n_layer=1, heavy_mode="uniform4")
         ctx = H.make_ctx(w, b_init=w.prompt)
         ctx.begin_sequence_batch(w.batch, w.prompt)
         ctx.set_budgets([w.prompt])                   # keep everything: scores are read back per token
