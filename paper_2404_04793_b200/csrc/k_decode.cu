@@ -307,7 +307,7 @@ static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
 
 // Which attention kernel serves a shape: grouped bf16 heads go to the tensor-core kernel,
 // everything else (fp32, one query head per KV head, shapes it does not cover) to the fp32-pipe
-// kernel.  SQ_DECODE_PATH=alu|mma overrides the choice (for A/B measurements).
+// kernel.  SQ_DECODE_PATH=alu|mma overrides the choice (mma also keeps wide groups off the tcgen05 kernel) (for A/B measurements).
 static int decode_path_override() {
   static int mode = -1;
   if (mode < 0) {
@@ -317,11 +317,17 @@ static int decode_path_override() {
   return mode;
 }
 
-cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, cudaStream_t s) {
+cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
+                          size_t q_rows, cudaStream_t s) {
   if (n_items <= 0) return cudaSuccess;
   const int ovr = decode_path_override();
   bool done = false;
-  if (dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
+  if (dtype == SQ_BF16 && ovr == 0 && a.group > 32) {
+    cudaError_t e = launch_decode_attn_tc(a, n_items, pool_bytes, q_rows, s);
+    if (e == cudaSuccess) done = true;
+    else if (e != cudaErrorNotSupported) return e;
+  }
+  if (!done && dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
     cudaError_t e = launch_decode_attn_mma(a, n_items, s);
     if (e == cudaSuccess) done = true;
     else if (e != cudaErrorNotSupported) return e;

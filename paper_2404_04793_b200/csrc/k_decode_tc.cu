@@ -1,0 +1,358 @@
+// Decode attention for wide multi-query groups (33..128 query heads per KV head, head_dim 64,
+// bf16) on the 5th-generation tensor cores.  With g = 71 (Falcon-shaped MQA) the step needs
+// g flop per byte of K/V -- hundreds of TFLOP/s at HBM speed -- so both contractions run as
+// tcgen05.mma with accumulators in tensor memory:
+//   S[128 head rows x 128 tokens] = Q K_tile^T        (Q, K tile in shared memory, K-major)
+//   O[128 head rows x 64]        += P V_tile           (P bf16 in shared memory, V tile MN-major)
+// One CTA per (layer, unit, split); per 128-token tile the roles are
+//   warp 0      TMA: K and V tiles into a ring of stages (128-byte swizzle, no multicast)
+//   warp 1      MMA issue; S is double-buffered so S(i+1) runs under the softmax of tile i
+//   warps 2..5  thread = one head row (TMEM lane): p = exp2(s*scale - m_ref) straight from the
+//               accumulator row, no shuffles; P is written to shared memory as the next A operand
+// The reference maximum m_ref of a row is only moved (and O, l rescaled through tcgen05.ld/st)
+// when a tile's maximum exceeds it by more than 2^16, which keeps every weight finite while
+// leaving the result that of the exact softmax.  Every barrier wait is bounded.
+#include "sq_decode_common.cuh"
+#include "sq_internal.h"
+#include "sq_tc.cuh"
+
+namespace sq {
+
+using namespace tc;
+
+namespace {
+constexpr int kD = 64;
+constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K or V tile, also one P sub-tile
+constexpr float kRescaleSlack = 16.f;     // log2 units
+constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+}  // namespace
+
+template <int STAGES>
+__global__ void __launch_bounds__(192, 1)
+    decode_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                          const __grid_constant__ CUtensorMap tm_v, DecodeArgs a, long long pool_row_base) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* q_s = smem;                               // [128 rows][64]
+  unsigned char* k_s = q_s + kTileBytes;                   // STAGES tiles
+  unsigned char* v_s = k_s + STAGES * kTileBytes;          // STAGES tiles
+  unsigned char* p_s = v_s + STAGES * kTileBytes;          // 2 buffers x 2 sub-tiles
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(p_s + 4 * kTileBytes);
+  static_assert(10 + 2 * STAGES <= 16, "barrier block");
+  const uint32_t bar_q = s_u32(bars + 0), bar_odone = s_u32(bars + 1);
+  auto bar_full = [&](int s) { return s_u32(bars + 2 + s); };
+  auto bar_empty = [&](int s) { return s_u32(bars + 2 + STAGES + s); };
+  auto bar_sfull = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + b); };
+  auto bar_sfree = [&](int b) { return s_u32(bars + 4 + 2 * STAGES + b); };
+  auto bar_pready = [&](int b) { return s_u32(bars + 6 + 2 * STAGES + b); };
+  auto bar_pfree = [&](int b) { return s_u32(bars + 8 + 2 * STAGES + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  ItemLoc it;
+  if (!locate(a, blockIdx.x, -1, it)) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const LayerDesc* ldp = a.layers + it.layer;
+  const int b = ldp->b, cap = ldp->cap, G = a.group;
+  const int unit = it.local / it.n_split, split = it.local - unit * it.n_split;
+  const int len = min(a.n_tok + 1, b);
+  const bool h2o = (a.policy == SQ_POLICY_H2O);
+  int w;
+  if (h2o) {
+    w = (a.n_tok < b) ? a.n_tok : reinterpret_cast<const int*>(a.pool + ldp->victim_off)[unit];
+    if (w < 0 || w >= b) {
+      if (tid == 0) atomicOr(a.status, 2);
+      w = 0;
+    }
+  } else {
+    w = ring_slot(a.n_tok, b, ldp->ring_base, ldp->ring_origin);
+  }
+  const int t0 = split * a.split_tokens, t1 = min(len, t0 + a.split_tokens);
+  const int n_tiles = (t1 - t0 + kTM - 1) / kTM;
+  const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
+  const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
+  using bf16 = __nv_bfloat16;
+  bf16* Kb = reinterpret_cast<bf16*>(a.pool + ldp->k_off) + (size_t)unit * cap * kD;
+  bf16* Vb = reinterpret_cast<bf16*>(a.pool + ldp->v_off) + (size_t)unit * cap * kD;
+  const bf16* kn = reinterpret_cast<const bf16*>(a.k_new) + (tok * a.n_kv_head + kvh) * kD;
+  const bf16* vn = reinterpret_cast<const bf16*>(a.v_new) + (tok * a.n_kv_head + kvh) * kD;
+  bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
+  float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
+  float* po = a.part_o + (size_t)blockIdx.x * G * kD;
+  // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q
+  const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap - pool_row_base;
+  const long long v_row0 = ldp->v_off / (kD * 2) + (long long)unit * cap - pool_row_base;
+  const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
+
+  // the CTA whose range holds slot w stores the new token first (generic proxy), then lets
+  // the TMA reads (async proxy) see it
+  if (w >= t0 && w < t1) {
+    if (tid < 16) {
+      const bool is_v = tid >= 8;
+      const int c = tid & 7;
+      const uint4 val = *reinterpret_cast<const uint4*>((is_v ? vn : kn) + c * 8);
+      *reinterpret_cast<uint4*>((is_v ? Vb : Kb) + (size_t)w * kD + c * 8) = val;
+    }
+    if (tid == 16) {
+      reinterpret_cast<int*>(a.pool + ldp->pos_off)[(size_t)unit * cap + w] = a.n_tok;
+      if (h2o) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
+    }
+    __threadfence();
+    fence_proxy_async();
+  }
+  if (tid == 0) {
+    mbar_init(bar_q, 1);
+    mbar_init(bar_odone, 1);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full(s), 1);
+      mbar_init(bar_empty(s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_sfull(i), 1);
+      mbar_init(bar_sfree(i), 128);
+      mbar_init(bar_pready(i), 128);
+      mbar_init(bar_pfree(i), 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_o = tmem_base + 256;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      mbar_expect_tx(bar_q, kTileBytes);
+      tma_load_2d(s_u32(q_s), &tm_q, 0, (int)q_row0, bar_q);
+      int issued = 0;
+      for (int i = 0; i < n_tiles; ++i) {
+        const int st = i % STAGES;
+        if (i >= STAGES && !mbar_wait(bar_empty(st), ((i / STAGES) - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(bar_full(st), 2 * kTileBytes);
+        tma_load_2d(s_u32(k_s + st * kTileBytes), &tm_k, 0, (int)(k_row0 + t0 + i * kTM), bar_full(st));
+        tma_load_2d(s_u32(v_s + st * kTileBytes), &tm_v, 0, (int)(v_row0 + t0 + i * kTM), bar_full(st));
+        issued = i + 1;
+      }
+      if (*abort_flag) {
+        mbar_wait(bar_q, 0, abort_flag);
+        for (int i = max(0, issued - STAGES); i < issued; ++i)
+          for (int k = 0; k < kSpinLimit && !mbar_try_wait(bar_full(i % STAGES), (i / STAGES) & 1); ++k) {
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    auto issue_s = [&](int i) -> bool {
+      const int st = i % STAGES, buf = i & 1;
+      if (!mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag)) return false;
+      if (i >= 2 && !mbar_wait(bar_sfree(buf), ((i >> 1) - 1) & 1, abort_flag)) return false;
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k)
+          umma_bf16(tmem_base + buf * kTM, umma_desc(s_u32(q_s) + k * 32), umma_desc(s_u32(k_s + st * kTileBytes) + k * 32),
+                    kIdescS, k > 0 ? 1u : 0u);
+        umma_commit(bar_sfull(buf));
+      }
+      __syncwarp();
+      return true;
+    };
+    bool ok = mbar_wait(bar_q, 0, abort_flag);
+    if (ok) ok = issue_s(0);
+    for (int i = 0; ok && i < n_tiles; ++i) {
+      if (i + 1 < n_tiles) ok = issue_s(i + 1);
+      if (!ok) break;
+      const int st = i % STAGES, pb = i & 1;
+      ok = mbar_wait(bar_pready(pb), (i >> 1) & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < kTM / 16; ++k) {
+          // A = P: K-major, 64-token sub-tiles; B = V: MN-major, 16 tokens = 2 KB per step
+          const uint32_t pa = s_u32(p_s + (pb * 2 + k / 4) * kTileBytes) + (k % 4) * 32;
+          const uint32_t vb = s_u32(v_s + st * kTileBytes) + k * 2048;
+          umma_bf16(tmem_o, umma_desc(pa), umma_desc(vb), kIdescO, (i > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(bar_empty(st));
+        umma_commit(bar_pfree(pb));
+        umma_commit(bar_odone);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------- softmax: thread = one head row ----------------
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const bool live = row < G;               // this lane's row is a real head
+    const bool warp_live = quarter * 32 < G;  // tcgen05.ld/st are warp-wide: whole warps opt in or out
+    const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+    float m_ref = -INFINITY, l_true = 0.f, l_w = 0.f;
+    bool ok = true;
+    for (int i = 0; ok && i < n_tiles; ++i) {
+      const int buf = i & 1, pb = i & 1, st = i % STAGES;
+      const int tile_row0 = t0 + i * kTM;
+      const int n_valid = min(kTM, t1 - tile_row0);
+      ok = mbar_wait(bar_sfull(buf), (i >> 1) & 1, abort_flag);
+      if (ok && i >= 2) ok = mbar_wait(bar_pfree(pb), ((i >> 1) - 1) & 1, abort_flag);
+      if (ok && n_valid < kTM) {
+        // rows of the V tile past the unit's last token may hold anything: zero them
+        ok = mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag);
+        if (ok && row >= n_valid) {
+          uint4* vrow = reinterpret_cast<uint4*>(v_s + st * kTileBytes + row * 128);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0, 0, 0, 0);
+        }
+      }
+      if (!ok) break;
+      tc_fence_after();
+      if (warp_live) {
+        // pass A: the row's maximum over the tile's valid tokens
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          tmem_ld32(tmem_base + lane_sel + buf * kTM + c * 32, v);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < n_valid) mx = fmaxf(mx, v[j]);
+        }
+        const float mx2 = mx * a.scale_log2;
+        const bool need = (i > 0) && (mx2 > m_ref + kRescaleSlack);
+        if (i == 0) m_ref = mx2;
+        if (__any_sync(0xffffffffu, need)) {
+          // rare: move the reference of the rows that need it; O (complete up to tile i-1) and
+          // the sums shrink with it.  The whole warp takes part in the TMEM round trip.
+          ok = mbar_wait(bar_odone, (i - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const float f = need ? ex2(m_ref - mx2) : 1.f;
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            float o[32];
+            tmem_ld32(tmem_o + lane_sel + c * 32, o);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] *= f;
+            tmem_st32(tmem_o + lane_sel + c * 32, o);
+          }
+          l_true *= f;
+          l_w *= f;
+          if (need) m_ref = mx2;
+        }
+        // pass B: weights, their sums, P as the next A operand
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          tmem_ld32(tmem_base + lane_sel + buf * kTM + c * 32, v);
+          if (h2o && live) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j < n_valid) logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = v[j] * a.scale_log2;
+          }
+          float sum = 0.f, sum_w = 0.f;
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float p0 = ex2(fmaf(v[j], a.scale_log2, -m_ref));
+            float p1 = ex2(fmaf(v[j + 1], a.scale_log2, -m_ref));
+            if (c * 32 + j >= n_valid) p0 = 0.f;
+            if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+            sum += p0 + p1;
+            const uint32_t u = pack2(p0, p1);
+            pk[j / 2] = u;
+            sum_w += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
+          }
+          l_true += sum;
+          l_w += sum_w;
+          // tokens c*32 .. c*32+31 of this row: four 16-byte chunks of P sub-tile (c / 2)
+          unsigned char* prow = p_s + (pb * 2 + (c >> 1)) * kTileBytes + row * 128;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int chunk = (c & 1) * 4 + q4;
+            *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
+                make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+          }
+        }
+      }
+      fence_proxy_async();  // P (and the zeroed V rows) must be visible to the tensor core
+      tc_fence_before();
+      mbar_arrive(bar_pready(pb));
+      mbar_arrive(bar_sfree(buf));
+    }
+    // ---------------- epilogue: O / l -> out (or the split-K partial) ----------------
+    if (ok) ok = mbar_wait(bar_odone, (n_tiles - 1) & 1, abort_flag);
+    if (ok && warp_live) {
+      tc_fence_after();
+      const float inv = 1.f / l_w;
+#pragma unroll 1
+      for (int c = 0; c < 2; ++c) {
+        float o[32];
+        tmem_ld32(tmem_o + lane_sel + c * 32, o);
+        if (!live) continue;
+        if (it.n_split == 1) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            *reinterpret_cast<uint4*>(ob + (size_t)row * kD + c * 32 + q4 * 8) =
+                make_uint4(pack2(o[q4 * 8] * inv, o[q4 * 8 + 1] * inv), pack2(o[q4 * 8 + 2] * inv, o[q4 * 8 + 3] * inv),
+                           pack2(o[q4 * 8 + 4] * inv, o[q4 * 8 + 5] * inv), pack2(o[q4 * 8 + 6] * inv, o[q4 * 8 + 7] * inv));
+        } else {
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<float4*>(po + (size_t)row * kD + c * 32 + q4 * 4) =
+                make_float4(o[q4 * 4], o[q4 * 4 + 1], o[q4 * 4 + 2], o[q4 * 4 + 3]);
+        }
+      }
+      if (live) {
+        stat[row * kStatStride] = m_ref;
+        stat[row * kStatStride + 1] = l_true;
+        stat[row * kStatStride + 2] = l_w;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+  if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
+}
+
+// Returns cudaErrorNotSupported when the shape is outside this kernel's range.
+cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s) {
+  constexpr int STAGES = 3;
+  if (a.head_dim != kD || a.group <= 32 || a.group > 128) return cudaErrorNotSupported;
+  const long long pool_rows = (long long)(pool_bytes / (kD * 2));
+  if (pool_rows + kTM > 0x7fffffffLL || (long long)q_rows + kTM > 0x7fffffffLL) return cudaErrorNotSupported;
+  CUtensorMap tm_q, tm_k, tm_v;
+  if (!make_tile_map(&tm_q, a.q, (long long)q_rows, kD, kTM) || !make_tile_map(&tm_k, a.pool, pool_rows, kD, kTM) ||
+      !make_tile_map(&tm_v, a.pool, pool_rows, kD, kTM))
+    return cudaErrorNotSupported;
+  constexpr size_t smem = 1024 + (size_t)(1 + 2 * STAGES + 4) * kTileBytes + 8 * 16 + 16;
+  auto kern = decode_attn_tc_kernel<STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kern<<<n_items, 192, smem, s>>>(tm_q, tm_k, tm_v, a, 0LL);
+  return cudaGetLastError();
+}
+
+}  // namespace sq

@@ -16,91 +16,12 @@
 // completion through tcgen05.commit -> mbarrier; warps 2-5 drain the accumulators with
 // tcgen05.ld.  Two accumulator buffers let the next tile's MMA run under this tile's exponentials.
 // Every mbarrier wait is bounded: on expiry the CTA raises a status bit and winds down.
-#include <cuda.h>
-
 #include "sq_internal.h"
+#include "sq_tc.cuh"
 
 namespace sq {
 
-namespace {
-
-constexpr int kTM = 128;                 // tile rows (TMEM lanes) and columns
-constexpr int kSubBytes = kTM * 128;     // one [128 rows x 64 bf16] swizzled sub-tile
-constexpr int kSpinLimit = 1 << 22;
-constexpr int kStatusTimeout = 16;
-
-__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Waits for the phase with the given parity, giving up after kSpinLimit polls or once another
-// role has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255) == 255 && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<unsigned long long>(tm)), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-// shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ unsigned long long umma_desc(uint32_t saddr) {
-  return (unsigned long long)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, unsigned long long adesc, unsigned long long bdesc,
-                                          uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
-      "%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-}  // namespace
+using namespace tc;
 
 // SWEEP 1: rows = queries, streamed tiles = keys; SWEEP 2: rows = keys, streamed tiles = queries.
 template <int D, int STAGES, int SWEEP>
@@ -331,25 +252,26 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [rows, d] bf16 row-major tensor, box = 128 rows x 64 columns, 128-byte swizzle
-static bool make_map(CUtensorMap* tm, const void* base, long long rows, int d) {
+namespace tc {
+bool make_tile_map(CUtensorMap* tm, const void* base, long long rows, int d, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)d * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)kTM};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+}  // namespace tc
 
 template <int D, int STAGES>
 static cudaError_t launch_tc_t(const ScoreArgs& a, int* status, cudaStream_t s) {
   CUtensorMap tm_q, tm_k;
   const long long q_rows = (long long)a.batch * a.n_q_head * a.prompt, k_rows = (long long)a.batch * a.n_kv_head * a.prompt;
   if (q_rows + kTM > 0x7fffffffLL) return cudaErrorNotSupported;  // TMA coordinates are 32-bit
-  if (!make_map(&tm_q, a.q, q_rows, D) || !make_map(&tm_k, a.k, k_rows, D)) return cudaErrorNotSupported;
+  if (!tc::make_tile_map(&tm_q, a.q, q_rows, D, kTM) || !tc::make_tile_map(&tm_k, a.k, k_rows, D, kTM)) return cudaErrorNotSupported;
   constexpr size_t smem = 1024 + (size_t)(1 + STAGES) * (D / 64) * kSubBytes + 8 * 16 + 16 + 2 * kTM * 4;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   const int n_tile = (a.prompt + kTM - 1) / kTM;

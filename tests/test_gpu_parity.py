@@ -226,7 +226,7 @@ def test_tiny_config_full_trajectory():
     (torch.float32, 64, 2, 2), (torch.float32, 128, 8, 2), (torch.bfloat16, 128, 4, 4),
     (torch.bfloat16, 128, 8, 2), (torch.bfloat16, 128, 16, 2), (torch.bfloat16, 64, 71, 1),
     (torch.bfloat16, 64, 6, 2), (torch.bfloat16, 128, 20, 1), (torch.bfloat16, 64, 48, 2),
-    (torch.bfloat16, 128, 40, 1)])
+    (torch.bfloat16, 128, 40, 1), (torch.bfloat16, 64, 40, 1), (torch.bfloat16, 64, 128, 1)])
 def test_decode_small_shapes(policy, dtype, head_dim, hq, hkv):
     w = small("dec", 19, policy=policy, dtype=dtype, head_dim=head_dim, n_q_head=hq, n_kv_head=hkv,
               heavy_mode="uniform4", steps=7)
@@ -246,6 +246,41 @@ def test_decode_split_k_long_context(policy):
     w = small("split", 21, policy=policy, dtype=torch.bfloat16, head_dim=128, n_q_head=8, n_kv_head=2, batch=1,
               n_layer=2, prompt=3000, steps=3, heavy_mode="zipf")
     _run_decode_and_compare(w, budgets=[2500, 1100], check_every_step=False)
+
+
+@pytest.mark.parametrize("policy", [synth.SLIDING_WINDOW, synth.STREAMING_LLM, synth.H2O])
+def test_decode_wide_mqa_long_context(policy):
+    # Falcon-shaped group (71 query heads on one KV head): several 128-token tiles, ragged tail,
+    # with and without split-K
+    w = small("mqa", 28, policy=policy, dtype=torch.bfloat16, head_dim=64, n_q_head=71, n_kv_head=1, batch=2,
+              n_layer=2, prompt=1500, steps=3, hidden=64, heavy_mode="zipf")
+    _run_decode_and_compare(w, budgets=[1300, 700], check_every_step=False)
+    w1 = w.replace(batch=1, prompt=2100, wid=29)
+    _run_decode_and_compare(w1, budgets=[2050, 300], check_every_step=False)
+
+
+def test_decode_wide_mqa_growing_logits():
+    """Keys late in the cache are far larger than the early ones, so the running reference of
+    the softmax has to move after the first tile."""
+    w = small("mqa_grow", 30, policy=synth.SLIDING_WINDOW, dtype=torch.bfloat16, head_dim=64, n_q_head=71,
+              n_kv_head=1, batch=1, n_layer=1, prompt=400, steps=2, hidden=64)
+    ctx = H.make_ctx(w, b_init=512)
+    ctx.begin_sequence_batch(1, w.prompt)
+    ctx.set_budgets([512])
+    _, k, v = synth.prompt_qkv(w, 0, DEV, need_q=False)
+    k = k.clone()
+    k[:, :, 130:260] *= 12.0
+    k[:, :, 260:] *= 30.0
+    ctx.prefill_compress(0, k, v)
+    u = O.UnitCache(O.SLIDING_WINDOW, 512)
+    u.prefill(H.f64(k[0, 0]), H.f64(v[0, 0]))
+    for t in range(w.steps):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, 1, q, kn, vn, out)
+        want = u.decode_step(H.f64(q[0, 0]), H.f64(kn[0, 0, 0]), H.f64(vn[0, 0, 0]))
+        assert np.max(np.abs(H.f64(out[0, 0]) - want)) <= H.TOL_OUT[w.dtype]
+    assert ctx.status() == 0
 
 
 def test_decode_budget_one_and_sinks_only_edge():
