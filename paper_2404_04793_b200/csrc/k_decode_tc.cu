@@ -2,16 +2,20 @@
 // bf16) on the 5th-generation tensor cores.  With g = 71 (Falcon-shaped MQA) the step needs
 // g flop per byte of K/V -- hundreds of TFLOP/s at HBM speed -- so both contractions run as
 // tcgen05.mma with accumulators in tensor memory:
-//   S[128 head rows x 128 tokens] = Q K_tile^T        (Q, K tile in shared memory, K-major)
-//   O[128 head rows x 64]        += P V_tile           (P bf16 in shared memory, V tile MN-major)
+//   S[head rows x 128 tokens] = Q K_tile^T      (Q, K tile in shared memory, K-major)
+//   O[head rows x 64]        += P V_tile         (P bf16 in shared memory, V tile MN-major)
+//   L[head rows]             += P 1              (row sums of the bf16 weights actually used)
 // One CTA per (layer, unit, split); per 128-token tile the roles are
 //   warp 0      TMA: K and V tiles into a ring of stages (128-byte swizzle, no multicast)
-//   warp 1      MMA issue; S is double-buffered so S(i+1) runs under the softmax of tile i
+//   warp 1      MMA issue
 //   warps 2..5  thread = one head row (TMEM lane): p = exp2(s*scale - m_ref) straight from the
-//               accumulator row, no shuffles; P is written to shared memory as the next A operand
-// The reference maximum m_ref of a row is only moved (and O, l rescaled through tcgen05.ld/st)
-// when a tile's maximum exceeds it by more than 2^16, which keeps every weight finite while
-// leaving the result that of the exact softmax.  Every barrier wait is bounded.
+//               accumulator row, no shuffles; P goes to shared memory as the next A operand
+// A row's reference m_ref is its maximum over the first tile; later tiles reuse it and only
+// when a weight would exceed 2^16 is the reference moved (O and the sums rescaled through
+// tcgen05.ld/st, the tile redone): every weight stays finite and the result is that of the
+// exact softmax.  Up to 96 heads the kernel keeps one accumulator buffer and a small footprint
+// so two CTAs share an SM; above that it double-buffers S in one CTA per SM.
+// Every barrier wait is bounded.
 #include "sq_decode_common.cuh"
 #include "sq_internal.h"
 #include "sq_tc.cuh"
@@ -22,37 +26,51 @@ using namespace tc;
 
 namespace {
 constexpr int kD = 64;
-constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K or V tile, also one P sub-tile
-constexpr float kRescaleSlack = 16.f;     // log2 units
-constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K or V tile
+constexpr int kOnesBytes = 2048;          // 16 rows x 128 B of bf16 ones (B operand of the row-sum MMA)
+constexpr float kMaxWeight = 65536.f;     // 2^16
+constexpr uint32_t idesc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 }  // namespace
 
-template <int STAGES>
-__global__ void __launch_bounds__(192, 1)
+// ROWS: head rows held in shared memory (96 or 128); NSB: accumulator / P buffers (1 or 2).
+template <int STAGES, int ROWS, int NSB, bool H2O>
+__global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
     decode_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                          const __grid_constant__ CUtensorMap tm_v, DecodeArgs a, long long pool_row_base) {
+                          const __grid_constant__ CUtensorMap tm_v, DecodeArgs a) {
+  constexpr int kQBytes = ROWS * 128;  // Q tile and one P sub-tile (64 tokens)
+  constexpr int kTmemCols = NSB == 1 ? 256 : 512;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* q_s = smem;                               // [128 rows][64]
-  unsigned char* k_s = q_s + kTileBytes;                   // STAGES tiles
-  unsigned char* v_s = k_s + STAGES * kTileBytes;          // STAGES tiles
-  unsigned char* p_s = v_s + STAGES * kTileBytes;          // 2 buffers x 2 sub-tiles
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(p_s + 4 * kTileBytes);
-  static_assert(10 + 2 * STAGES <= 16, "barrier block");
+  // The MMAs address 128 rows of Q and P; with ROWS = 96 rows 96..127 alias the bytes that
+  // follow (rows are independent, those accumulator rows are never read).
+  unsigned char* q_s = smem;
+  unsigned char* p_s = q_s + kQBytes;                       // NSB x 2 sub-tiles
+  unsigned char* k_s = p_s + NSB * 2 * kQBytes;             // STAGES tiles
+  unsigned char* v_s = k_s + STAGES * kTileBytes;           // STAGES tiles
+  unsigned char* ones_s = v_s + STAGES * kTileBytes;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(ones_s + kOnesBytes);
+  static_assert(2 + 2 * STAGES + 4 * NSB <= 16, "barrier block");
   const uint32_t bar_q = s_u32(bars + 0), bar_odone = s_u32(bars + 1);
   auto bar_full = [&](int s) { return s_u32(bars + 2 + s); };
   auto bar_empty = [&](int s) { return s_u32(bars + 2 + STAGES + s); };
   auto bar_sfull = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + b); };
-  auto bar_sfree = [&](int b) { return s_u32(bars + 4 + 2 * STAGES + b); };
-  auto bar_pready = [&](int b) { return s_u32(bars + 6 + 2 * STAGES + b); };
-  auto bar_pfree = [&](int b) { return s_u32(bars + 8 + 2 * STAGES + b); };
+  auto bar_sfree = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + NSB + b); };
+  auto bar_pready = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + 2 * NSB + b); };
+  auto bar_pfree = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + 3 * NSB + b); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -63,9 +81,8 @@ __global__ void __launch_bounds__(192, 1)
   const int b = ldp->b, cap = ldp->cap, G = a.group;
   const int unit = it.local / it.n_split, split = it.local - unit * it.n_split;
   const int len = min(a.n_tok + 1, b);
-  const bool h2o = (a.policy == SQ_POLICY_H2O);
   int w;
-  if (h2o) {
+  if (H2O) {
     w = (a.n_tok < b) ? a.n_tok : reinterpret_cast<const int*>(a.pool + ldp->victim_off)[unit];
     if (w < 0 || w >= b) {
       if (tid == 0) atomicOr(a.status, 2);
@@ -88,8 +105,8 @@ __global__ void __launch_bounds__(192, 1)
   float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
   float* po = a.part_o + (size_t)blockIdx.x * G * kD;
   // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q
-  const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap - pool_row_base;
-  const long long v_row0 = ldp->v_off / (kD * 2) + (long long)unit * cap - pool_row_base;
+  const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
+  const long long v_row0 = ldp->v_off / (kD * 2) + (long long)unit * cap;
   const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
 
   // the CTA whose range holds slot w stores the new token first (generic proxy), then lets
@@ -103,9 +120,13 @@ __global__ void __launch_bounds__(192, 1)
     }
     if (tid == 16) {
       reinterpret_cast<int*>(a.pool + ldp->pos_off)[(size_t)unit * cap + w] = a.n_tok;
-      if (h2o) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
+      if (H2O) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
     }
     __threadfence();
+    fence_proxy_async();
+  }
+  if (tid >= 64 && tid < 64 + kOnesBytes / 16) {
+    reinterpret_cast<uint4*>(ones_s)[tid - 64] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
     fence_proxy_async();
   }
   if (tid == 0) {
@@ -115,7 +136,7 @@ __global__ void __launch_bounds__(192, 1)
       mbar_init(bar_full(s), 1);
       mbar_init(bar_empty(s), 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NSB; ++i) {
       mbar_init(bar_sfull(i), 1);
       mbar_init(bar_sfree(i), 128);
       mbar_init(bar_pready(i), 128);
@@ -125,19 +146,20 @@ __global__ void __launch_bounds__(192, 1)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "n"(kTmemCols)
+                 : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_o = tmem_base + 256;
+  const uint32_t tmem_o = tmem_base + NSB * kTM;  // 64 output columns, then 16 columns of row sums
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      mbar_expect_tx(bar_q, kTileBytes);
+      mbar_expect_tx(bar_q, kQBytes);
       tma_load_2d(s_u32(q_s), &tm_q, 0, (int)q_row0, bar_q);
       int issued = 0;
       for (int i = 0; i < n_tiles; ++i) {
@@ -158,15 +180,15 @@ __global__ void __launch_bounds__(192, 1)
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     auto issue_s = [&](int i) -> bool {
-      const int st = i % STAGES, buf = i & 1;
+      const int st = i % STAGES, buf = i % NSB;
       if (!mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag)) return false;
-      if (i >= 2 && !mbar_wait(bar_sfree(buf), ((i >> 1) - 1) & 1, abort_flag)) return false;
+      if (i >= NSB && !mbar_wait(bar_sfree(buf), ((i / NSB) - 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (lane == 0) {
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k)
           umma_bf16(tmem_base + buf * kTM, umma_desc(s_u32(q_s) + k * 32), umma_desc(s_u32(k_s + st * kTileBytes) + k * 32),
-                    kIdescS, k > 0 ? 1u : 0u);
+                    idesc(128, false), k > 0 ? 1u : 0u);
         umma_commit(bar_sfull(buf));
       }
       __syncwarp();
@@ -177,17 +199,19 @@ __global__ void __launch_bounds__(192, 1)
     for (int i = 0; ok && i < n_tiles; ++i) {
       if (i + 1 < n_tiles) ok = issue_s(i + 1);
       if (!ok) break;
-      const int st = i % STAGES, pb = i & 1;
-      ok = mbar_wait(bar_pready(pb), (i >> 1) & 1, abort_flag);
+      const int st = i % STAGES, pb = i % NSB;
+      ok = mbar_wait(bar_pready(pb), (i / NSB) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
+        const uint32_t acc = (i > 0) ? 1u : 0u;
 #pragma unroll
         for (int k = 0; k < kTM / 16; ++k) {
           // A = P: K-major, 64-token sub-tiles; B = V: MN-major, 16 tokens = 2 KB per step
-          const uint32_t pa = s_u32(p_s + (pb * 2 + k / 4) * kTileBytes) + (k % 4) * 32;
+          const uint32_t pa = s_u32(p_s + (pb * 2 + k / 4) * kQBytes) + (k % 4) * 32;
           const uint32_t vb = s_u32(v_s + st * kTileBytes) + k * 2048;
-          umma_bf16(tmem_o, umma_desc(pa), umma_desc(vb), kIdescO, (i > 0 || k > 0) ? 1u : 0u);
+          umma_bf16(tmem_o, umma_desc(pa), umma_desc(vb), idesc(kD, true), (k > 0) ? 1u : acc);
+          umma_bf16(tmem_o + kD, umma_desc(pa), umma_desc(s_u32(ones_s)), idesc(16, false), (k > 0) ? 1u : acc);
         }
         umma_commit(bar_empty(st));
         umma_commit(bar_pfree(pb));
@@ -199,17 +223,75 @@ __global__ void __launch_bounds__(192, 1)
     // ---------------- softmax: thread = one head row ----------------
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const bool live = row < G;               // this lane's row is a real head
+    const bool live = row < G;                // this lane's row is a real head
     const bool warp_live = quarter * 32 < G;  // tcgen05.ld/st are warp-wide: whole warps opt in or out
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-    float m_ref = -INFINITY, l_true = 0.f, l_w = 0.f;
+    float m_ref = -INFINITY, l_true = 0.f;
     bool ok = true;
+
+    // Row maximum of the tile's valid tokens, in the log2 domain.
+    auto tile_max = [&](uint32_t s_addr, int n_valid) {
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(s_addr + c * 32, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c * 32 + j < n_valid) mx = fmaxf(mx, v[j]);
+      }
+      return mx * a.scale_log2;
+    };
+    // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to shared memory, the fp32 sum of the
+    // weights to *sum (H2O only), logits to global (H2O only); returns the largest weight.
+    auto tile_weights = [&](uint32_t s_addr, int pb, int tile_row0, int n_valid, float* sum) {
+      uint32_t pmax = 0u;
+      float acc = 0.f;
+      const bool full = (n_valid == kTM);
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(s_addr + c * 32, v);
+        if (H2O && live) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < n_valid) logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = v[j] * a.scale_log2;
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          float p0 = ex2(fmaf(v[j], a.scale_log2, -m_ref));
+          float p1 = ex2(fmaf(v[j + 1], a.scale_log2, -m_ref));
+          if (!full) {
+            if (c * 32 + j >= n_valid) p0 = 0.f;
+            if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+          }
+          if (H2O) acc += p0 + p1;
+          pk[j / 2] = pack2(p0, p1);
+          pmax = max_bf16x2(pmax, pk[j / 2]);
+        }
+        // tokens c*32 .. c*32+31 of this row: four 16-byte chunks of P sub-tile (c / 2)
+        if (row < ROWS) {
+          unsigned char* prow = p_s + (pb * 2 + (c >> 1)) * kQBytes + row * 128;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int chunk = (c & 1) * 4 + q4;
+            *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
+                make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+          }
+        }
+      }
+      *sum = acc;
+      return fmaxf(__uint_as_float(pmax << 16), __uint_as_float(pmax & 0xffff0000u));
+    };
+
     for (int i = 0; ok && i < n_tiles; ++i) {
-      const int buf = i & 1, pb = i & 1, st = i % STAGES;
+      const int buf = i % NSB, pb = i % NSB, st = i % STAGES;
       const int tile_row0 = t0 + i * kTM;
       const int n_valid = min(kTM, t1 - tile_row0);
-      ok = mbar_wait(bar_sfull(buf), (i >> 1) & 1, abort_flag);
-      if (ok && i >= 2) ok = mbar_wait(bar_pfree(pb), ((i >> 1) - 1) & 1, abort_flag);
+      const uint32_t s_addr = tmem_base + lane_sel + buf * kTM;
+      ok = mbar_wait(bar_sfull(buf), (i / NSB) & 1, abort_flag);
+      if (ok && i >= NSB) ok = mbar_wait(bar_pfree(pb), ((i / NSB) - 1) & 1, abort_flag);
       if (ok && n_valid < kTM) {
         // rows of the V tile past the unit's last token may hold anything: zero them
         ok = mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag);
@@ -222,28 +304,21 @@ __global__ void __launch_bounds__(192, 1)
       if (!ok) break;
       tc_fence_after();
       if (warp_live) {
-        // pass A: the row's maximum over the tile's valid tokens
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          float v[32];
-          tmem_ld32(tmem_base + lane_sel + buf * kTM + c * 32, v);
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < n_valid) mx = fmaxf(mx, v[j]);
-        }
-        const float mx2 = mx * a.scale_log2;
-        const bool need = (i > 0) && (mx2 > m_ref + kRescaleSlack);
-        if (i == 0) m_ref = mx2;
-        if (__any_sync(0xffffffffu, need)) {
-          // rare: move the reference of the rows that need it; O (complete up to tile i-1) and
-          // the sums shrink with it.  The whole warp takes part in the TMEM round trip.
+        if (i == 0) m_ref = tile_max(s_addr, n_valid);
+        float sum;
+        float pmax = tile_weights(s_addr, pb, tile_row0, n_valid, &sum);
+        if (__any_sync(0xffffffffu, pmax > kMaxWeight)) {
+          // rare: move the reference of the rows that need it; O and the sums (complete up to
+          // tile i-1) shrink with it, then the tile is redone.  The whole warp takes part in
+          // the TMEM round trip.
+          const float mx2 = tile_max(s_addr, n_valid);
+          const bool need = pmax > kMaxWeight;
           ok = mbar_wait(bar_odone, (i - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_ref - mx2) : 1.f;
 #pragma unroll 1
-          for (int c = 0; c < 2; ++c) {
+          for (int c = 0; c < 3; ++c) {
             float o[32];
             tmem_ld32(tmem_o + lane_sel + c * 32, o);
 #pragma unroll
@@ -251,57 +326,26 @@ __global__ void __launch_bounds__(192, 1)
             tmem_st32(tmem_o + lane_sel + c * 32, o);
           }
           l_true *= f;
-          l_w *= f;
           if (need) m_ref = mx2;
+          pmax = tile_weights(s_addr, pb, tile_row0, n_valid, &sum);
         }
-        // pass B: weights, their sums, P as the next A operand
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          float v[32];
-          tmem_ld32(tmem_base + lane_sel + buf * kTM + c * 32, v);
-          if (h2o && live) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c * 32 + j < n_valid) logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = v[j] * a.scale_log2;
-          }
-          float sum = 0.f, sum_w = 0.f;
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float p0 = ex2(fmaf(v[j], a.scale_log2, -m_ref));
-            float p1 = ex2(fmaf(v[j + 1], a.scale_log2, -m_ref));
-            if (c * 32 + j >= n_valid) p0 = 0.f;
-            if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
-            sum += p0 + p1;
-            const uint32_t u = pack2(p0, p1);
-            pk[j / 2] = u;
-            sum_w += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
-          }
-          l_true += sum;
-          l_w += sum_w;
-          // tokens c*32 .. c*32+31 of this row: four 16-byte chunks of P sub-tile (c / 2)
-          unsigned char* prow = p_s + (pb * 2 + (c >> 1)) * kTileBytes + row * 128;
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int chunk = (c & 1) * 4 + q4;
-            *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
-                make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
-          }
-        }
+        l_true += sum;
       }
       fence_proxy_async();  // P (and the zeroed V rows) must be visible to the tensor core
       tc_fence_before();
       mbar_arrive(bar_pready(pb));
       mbar_arrive(bar_sfree(buf));
     }
-    // ---------------- epilogue: O / l -> out (or the split-K partial) ----------------
+    // ---------------- epilogue: O / L -> out (or the split-K partial) ----------------
     if (ok) ok = mbar_wait(bar_odone, (n_tiles - 1) & 1, abort_flag);
     if (ok && warp_live) {
       tc_fence_after();
+      float o[32];
+      tmem_ld32(tmem_o + lane_sel + 2 * 32, o);
+      const float l_w = o[0];  // sum of the bf16 weights that went into O
       const float inv = 1.f / l_w;
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
-        float o[32];
         tmem_ld32(tmem_o + lane_sel + c * 32, o);
         if (!live) continue;
         if (it.n_split == 1) {
@@ -319,7 +363,7 @@ __global__ void __launch_bounds__(192, 1)
       }
       if (live) {
         stat[row * kStatStride] = m_ref;
-        stat[row * kStatStride + 1] = l_true;
+        stat[row * kStatStride + 1] = H2O ? l_true : l_w;
         stat[row * kStatStride + 2] = l_w;
       }
     }
@@ -328,31 +372,42 @@ __global__ void __launch_bounds__(192, 1)
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
 }
 
-// Returns cudaErrorNotSupported when the shape is outside this kernel's range.
-cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s) {
-  constexpr int STAGES = 3;
-  if (a.head_dim != kD || a.group <= 32 || a.group > 128) return cudaErrorNotSupported;
-  const long long pool_rows = (long long)(pool_bytes / (kD * 2));
-  if (pool_rows + kTM > 0x7fffffffLL || (long long)q_rows + kTM > 0x7fffffffLL) return cudaErrorNotSupported;
-  CUtensorMap tm_q, tm_k, tm_v;
-  if (!make_tile_map(&tm_q, a.q, (long long)q_rows, kD, kTM) || !make_tile_map(&tm_k, a.pool, pool_rows, kD, kTM) ||
-      !make_tile_map(&tm_v, a.pool, pool_rows, kD, kTM))
-    return cudaErrorNotSupported;
-  constexpr size_t smem = 1024 + (size_t)(1 + 2 * STAGES + 4) * kTileBytes + 8 * 16 + 16;
-  auto kern = decode_attn_tc_kernel<STAGES>;
+template <int STAGES, int ROWS, int NSB, bool H2O>
+static cudaError_t launch_tc_cfg(const DecodeArgs& a, int n_items, const CUtensorMap& tq, const CUtensorMap& tk,
+                                 const CUtensorMap& tv, cudaStream_t s) {
+  constexpr size_t smem = 1024 + (size_t)ROWS * 128 * (1 + 2 * NSB) + (size_t)2 * STAGES * kTileBytes + kOnesBytes + 8 * 16 + 16;
+  auto kern = decode_attn_tc_kernel<STAGES, ROWS, NSB, H2O>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<n_items, 192, smem, s>>>(tm_q, tm_k, tm_v, a, 0LL);
+  kern<<<n_items, 192, smem, s>>>(tq, tk, tv, a);
   return cudaGetLastError();
+}
+
+// Returns cudaErrorNotSupported when the shape is outside this kernel's range.
+cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s) {
+  if (a.head_dim != kD || a.group <= 32 || a.group > 128) return cudaErrorNotSupported;
+  const long long pool_rows = (long long)(pool_bytes / (kD * 2));
+  if (pool_rows + kTM > 0x7fffffffLL || (long long)q_rows + kTM > 0x7fffffffLL) return cudaErrorNotSupported;
+  const int rows = a.group <= 96 ? 96 : 128;
+  CUtensorMap tm_q, tm_k, tm_v;
+  if (!make_tile_map(&tm_q, a.q, (long long)q_rows, kD, rows) || !make_tile_map(&tm_k, a.pool, pool_rows, kD, kTM) ||
+      !make_tile_map(&tm_v, a.pool, pool_rows, kD, kTM))
+    return cudaErrorNotSupported;
+  const bool h2o = a.policy == SQ_POLICY_H2O;
+  if (rows == 96)
+    return h2o ? launch_tc_cfg<2, 96, 1, true>(a, n_items, tm_q, tm_k, tm_v, s)
+               : launch_tc_cfg<2, 96, 1, false>(a, n_items, tm_q, tm_k, tm_v, s);
+  return h2o ? launch_tc_cfg<3, 128, 2, true>(a, n_items, tm_q, tm_k, tm_v, s)
+             : launch_tc_cfg<3, 128, 2, false>(a, n_items, tm_q, tm_k, tm_v, s);
 }
 
 }  // namespace sq
