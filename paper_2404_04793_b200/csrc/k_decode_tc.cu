@@ -29,7 +29,7 @@ constexpr int kD = 64;
 constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K or V tile
 constexpr int kOnesBytes = 2048;          // 16 rows x 128 B of bf16 ones (B operand of the row-sum MMA)
 constexpr float kMaxWeight = 65536.f;     // 2^16
-constexpr uint32_t idesc(int n, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t idesc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(128 >> 4) << 24);
 }
