@@ -1,0 +1,106 @@
+"""Decode-step micro-benchmark: times sq_decode_step alone on any workload shape.
+
+    python -m paper_2404_04793_b200.microbench --workload falcon_7b --batch 32 --prompt 8192 \
+        --budget-pct 30 --policy sliding_window --steps 12 [--per-layer]
+
+The cache is filled through the regular calls (importance on a 256-token slice per layer,
+allocation, prefill compression of one random prompt reused for every layer; H2O prompts get
+random scores), so only the decode inputs are large.  Prints one JSON line with the step time
+and the achieved K/V bandwidth.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import engine, synth
+
+POLICIES = {"sliding_window": synth.SLIDING_WINDOW, "streaming_llm": synth.STREAMING_LLM, "h2o": synth.H2O}
+
+
+def build_workload(args) -> synth.Workload:
+    if args.workload == "falcon_7b":
+        w = synth.falcon_7b(args.batch or 32, args.prompt or 2048, args.budget_pct or 20.0,
+                            POLICIES[args.policy] if args.policy else synth.SLIDING_WINDOW)
+    else:
+        w = synth.WORKLOADS[args.workload]()
+        kw = {}
+        if args.batch:
+            kw["batch"] = args.batch
+        if args.prompt:
+            kw["prompt"] = args.prompt
+        if args.budget_pct:
+            kw["budget_pct"] = args.budget_pct
+        if args.policy:
+            kw["policy"] = POLICIES[args.policy]
+        if kw:
+            w = w.replace(**kw)
+    return w
+
+
+def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, device="cuda:0"):
+    job = engine.Job(w.replace(steps=steps + warmup), device)
+    ctx = job.ctx
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    for l in range(w.n_layer):
+        a, b = synth.hidden_pair(w, l, device, batch=1, n_tok=256)
+        ctx.layer_importance(l, a, b)
+    ctx.allocate_budgets(w.b_init, w.p)
+    budgets, _ = ctx.get_budgets()
+    g = torch.Generator(device=device).manual_seed(1)
+    shape_kv = (w.batch, w.n_kv_head, w.prompt, w.head_dim)
+    k = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    v = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    acc = torch.rand(w.batch, w.n_kv_head, w.prompt, generator=g, device=device) if w.policy == synth.H2O else None
+    for l in range(w.n_layer):
+        ctx.prefill_compress(l, k, v, None, acc)
+    q = torch.randn(w.n_layer, w.batch, w.n_q_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    kn = torch.randn(w.n_layer, w.batch, w.n_kv_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    vn = torch.randn(w.n_layer, w.batch, w.n_kv_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    out = torch.empty_like(q)
+
+    def step():
+        if per_layer:
+            for l in range(w.n_layer):
+                ctx.decode_step(l, l + 1, q[l], kn[l], vn[l], out[l])
+        else:
+            ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    kv = w.batch * w.n_kv_head * sum(min(w.prompt + 1, b) for b in budgets) * 2 * w.head_dim * e
+    io = w.batch * w.n_layer * (2 * w.n_q_head + 2 * w.n_kv_head) * w.head_dim * e
+    extra = (w.batch * w.n_kv_head * sum(budgets) * 8) if w.policy == synth.H2O else 0
+    gbs = (kv + io + extra) / ms / 1e6
+    return dict(workload=w.name, per_layer=per_layer, ms_per_step=round(ms, 4), GBs=round(gbs, 1),
+                kv_GB=round(kv / 1e9, 3), algorithmic_bytes=kv + io + extra, tokens_per_s=round(w.batch / ms * 1e3),
+                flops=4 * w.n_q_head * w.head_dim * w.batch * sum(budgets), device_status=ctx.status())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="llama2_7b")
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--prompt", type=int, default=0)
+    ap.add_argument("--budget-pct", type=float, default=0.0)
+    ap.add_argument("--policy", default="")
+    ap.add_argument("--steps", type=int, default=12)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--per-layer", action="store_true")
+    args = ap.parse_args()
+    print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer)), flush=True)
+
+
+if __name__ == "__main__":
+    main()
