@@ -13,7 +13,7 @@ from ctypes import POINTER, byref, c_char_p, c_double, c_float, c_int32, c_int64
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libsq.so")
+LIB_PATH = os.environ.get("SQ_LIB_PATH") or os.path.join(_PKG, "libsq.so")
 
 SQ_OK, SQ_ERR_INVALID_ARG, SQ_ERR_STATE, SQ_ERR_CAPACITY, SQ_ERR_CUDA, SQ_ERR_UNSUPPORTED = range(6)
 SQ_POLICY_SLIDING_WINDOW, SQ_POLICY_STREAMING_LLM, SQ_POLICY_H2O = 0, 1, 2

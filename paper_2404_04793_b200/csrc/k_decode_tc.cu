@@ -3,19 +3,20 @@
 // g flop per byte of K/V -- hundreds of TFLOP/s at HBM speed -- so both contractions run as
 // tcgen05.mma with accumulators in tensor memory:
 //   S[head rows x 128 tokens] = Q K_tile^T      (Q, K tile in shared memory, K-major)
-//   O[head rows x 64]        += P V_tile         (P bf16 in shared memory, V tile MN-major)
-//   L[head rows]             += P 1              (row sums of the bf16 weights actually used)
-// One CTA per (layer, unit, split); per 128-token tile the roles are
+//   O[head rows x 64]        += P V_tile         (P bf16 in TENSOR memory, V tile MN-major)
+// One CTA per (layer, unit, split), two CTAs per SM; per 128-token tile the roles are
 //   warp 0      TMA: K and V tiles into a ring of stages (128-byte swizzle, no multicast)
 //   warp 1      MMA issue
 //   warps 2..5  thread = one head row (TMEM lane): p = exp2(s*scale - m_ref) straight from the
-//               accumulator row, no shuffles; P goes to shared memory as the next A operand
+//               accumulator row, no shuffles; P is packed to bf16 and stored back to tensor
+//               memory as the A operand of the second MMA
+// Measured on B200: one M=128, K=16 MMA costs 45-48 cycles for N <= 64 and 64 cycles for N = 128,
+// and operands read from shared memory compete with the TMA writes for its 128 B/clk; keeping P
+// in tensor memory (64 columns) removes 56 KB of shared-memory traffic per tile.
 // A row's reference m_ref is its maximum over the first tile; later tiles reuse it and only
 // when a weight would exceed 2^16 is the reference moved (O and the sums rescaled through
 // tcgen05.ld/st, the tile redone): every weight stays finite and the result is that of the
-// exact softmax.  Up to 96 heads the kernel keeps one accumulator buffer and a small footprint
-// so two CTAs share an SM; above that it double-buffers S in one CTA per SM.
-// Every barrier wait is bounded.
+// exact softmax.  Every barrier wait is bounded.
 #include "sq_decode_common.cuh"
 #include "sq_internal.h"
 #include "sq_tc.cuh"
@@ -27,13 +28,12 @@ using namespace tc;
 namespace {
 constexpr int kD = 64;
 constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K or V tile
-constexpr int kOnesBytes = 2048;          // 16 rows x 128 B of bf16 ones (B operand of the row-sum MMA)
 constexpr float kMaxWeight = 65536.f;     // 2^16
+constexpr int kColS = 0, kColP = 128, kColO = 192, kTmemCols = 256;
 __host__ __device__ constexpr uint32_t idesc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(128 >> 4) << 24);
 }
-
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -46,31 +46,25 @@ __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
 }
 }  // namespace
 
-// ROWS: head rows held in shared memory (96 or 128); NSB: accumulator / P buffers (1 or 2).
-template <int STAGES, int ROWS, int NSB, bool H2O>
-__global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
+// ROWS: head rows of Q held in shared memory (96 or 128).
+template <int STAGES, int ROWS, bool H2O>
+__global__ void __launch_bounds__(192, 2)
     decode_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, DecodeArgs a) {
-  constexpr int kQBytes = ROWS * 128;  // Q tile and one P sub-tile (64 tokens)
-  constexpr int kTmemCols = NSB == 1 ? 256 : 512;
+  constexpr int kQBytes = ROWS * 128;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  // The MMAs address 128 rows of Q and P; with ROWS = 96 rows 96..127 alias the bytes that
-  // follow (rows are independent, those accumulator rows are never read).
+  // The first MMA addresses 128 rows of Q; with ROWS = 96 rows 96..127 alias the K stage that
+  // follows (rows are independent, those accumulator rows are never read).
   unsigned char* q_s = smem;
-  unsigned char* p_s = q_s + kQBytes;                       // NSB x 2 sub-tiles
-  unsigned char* k_s = p_s + NSB * 2 * kQBytes;             // STAGES tiles
-  unsigned char* v_s = k_s + STAGES * kTileBytes;           // STAGES tiles
-  unsigned char* ones_s = v_s + STAGES * kTileBytes;
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(ones_s + kOnesBytes);
-  static_assert(2 + 2 * STAGES + 4 * NSB <= 16, "barrier block");
-  const uint32_t bar_q = s_u32(bars + 0), bar_odone = s_u32(bars + 1);
-  auto bar_full = [&](int s) { return s_u32(bars + 2 + s); };
-  auto bar_empty = [&](int s) { return s_u32(bars + 2 + STAGES + s); };
-  auto bar_sfull = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + b); };
-  auto bar_sfree = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + NSB + b); };
-  auto bar_pready = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + 2 * NSB + b); };
-  auto bar_pfree = [&](int b) { return s_u32(bars + 2 + 2 * STAGES + 3 * NSB + b); };
+  unsigned char* k_s = q_s + kQBytes;              // STAGES tiles
+  unsigned char* v_s = k_s + STAGES * kTileBytes;  // STAGES tiles
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(v_s + STAGES * kTileBytes);
+  static_assert(6 + 2 * STAGES <= 16, "barrier block");
+  const uint32_t bar_q = s_u32(bars + 0), bar_odone = s_u32(bars + 1), bar_sfull = s_u32(bars + 2),
+                 bar_sfree = s_u32(bars + 3), bar_pready = s_u32(bars + 4), bar_pfree = s_u32(bars + 5);
+  auto bar_full = [&](int s) { return s_u32(bars + 6 + s); };
+  auto bar_empty = [&](int s) { return s_u32(bars + 6 + STAGES + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -125,22 +119,16 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
     __threadfence();
     fence_proxy_async();
   }
-  if (tid >= 64 && tid < 64 + kOnesBytes / 16) {
-    reinterpret_cast<uint4*>(ones_s)[tid - 64] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
-    fence_proxy_async();
-  }
   if (tid == 0) {
     mbar_init(bar_q, 1);
     mbar_init(bar_odone, 1);
+    mbar_init(bar_sfull, 1);
+    mbar_init(bar_sfree, 4);   // one arrival per softmax warp
+    mbar_init(bar_pready, 4);
+    mbar_init(bar_pfree, 1);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full(s), 1);
       mbar_init(bar_empty(s), 1);
-    }
-    for (int i = 0; i < NSB; ++i) {
-      mbar_init(bar_sfull(i), 1);
-      mbar_init(bar_sfree(i), 128);
-      mbar_init(bar_pready(i), 128);
-      mbar_init(bar_pfree(i), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -154,7 +142,6 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_o = tmem_base + NSB * kTM;  // 64 output columns, then 16 columns of row sums
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -179,17 +166,19 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
+    const uint32_t q_addr = s_u32(q_s);
     auto issue_s = [&](int i) -> bool {
-      const int st = i % STAGES, buf = i % NSB;
+      const int st = i % STAGES;
       if (!mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag)) return false;
-      if (i >= NSB && !mbar_wait(bar_sfree(buf), ((i / NSB) - 1) & 1, abort_flag)) return false;
+      if (i >= 1 && !mbar_wait(bar_sfree, (i - 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (lane == 0) {
+        const uint32_t k_addr = s_u32(k_s + st * kTileBytes);
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k)
-          umma_bf16(tmem_base + buf * kTM, umma_desc(s_u32(q_s) + k * 32), umma_desc(s_u32(k_s + st * kTileBytes) + k * 32),
-                    idesc(128, false), k > 0 ? 1u : 0u);
-        umma_commit(bar_sfull(buf));
+          umma_bf16(tmem_base + kColS, umma_desc(q_addr + k * 32), umma_desc(k_addr + k * 32), idesc(128, false),
+                    k > 0 ? 1u : 0u);
+        umma_commit(bar_sfull);
       }
       __syncwarp();
       return true;
@@ -199,22 +188,19 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
     for (int i = 0; ok && i < n_tiles; ++i) {
       if (i + 1 < n_tiles) ok = issue_s(i + 1);
       if (!ok) break;
-      const int st = i % STAGES, pb = i % NSB;
-      ok = mbar_wait(bar_pready(pb), (i / NSB) & 1, abort_flag);
+      const int st = i % STAGES;
+      ok = mbar_wait(bar_pready, i & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
-        const uint32_t acc = (i > 0) ? 1u : 0u;
+        const uint32_t v_addr = s_u32(v_s + st * kTileBytes);
 #pragma unroll
-        for (int k = 0; k < kTM / 16; ++k) {
-          // A = P: K-major, 64-token sub-tiles; B = V: MN-major, 16 tokens = 2 KB per step
-          const uint32_t pa = s_u32(p_s + (pb * 2 + k / 4) * kQBytes) + (k % 4) * 32;
-          const uint32_t vb = s_u32(v_s + st * kTileBytes) + k * 2048;
-          umma_bf16(tmem_o, umma_desc(pa), umma_desc(vb), idesc(kD, true), (k > 0) ? 1u : acc);
-          umma_bf16(tmem_o + kD, umma_desc(pa), umma_desc(s_u32(ones_s)), idesc(16, false), (k > 0) ? 1u : acc);
-        }
+        for (int k = 0; k < kTM / 16; ++k)
+          // A = P in tensor memory: 16 tokens = 8 columns per step; B = V, MN-major: 2 KB per step
+          umma_bf16_ta(tmem_base + kColO, tmem_base + kColP + k * 8, umma_desc(v_addr + k * 2048), idesc(kD, true),
+                       (i > 0 || k > 0) ? 1u : 0u);
         umma_commit(bar_empty(st));
-        umma_commit(bar_pfree(pb));
+        umma_commit(bar_pfree);
         umma_commit(bar_odone);
       }
       __syncwarp();
@@ -226,11 +212,13 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
     const bool live = row < G;                // this lane's row is a real head
     const bool warp_live = quarter * 32 < G;  // tcgen05.ld/st are warp-wide: whole warps opt in or out
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-    float m_ref = -INFINITY, l_true = 0.f;
+    const uint32_t s_addr = tmem_base + lane_sel + kColS, p_addr = tmem_base + lane_sel + kColP,
+                   o_addr = tmem_base + lane_sel + kColO;
+    float m_ref = -INFINITY, l_true = 0.f, l_w = 0.f;
     bool ok = true;
 
     // Row maximum of the tile's valid tokens, in the log2 domain.
-    auto tile_max = [&](uint32_t s_addr, int n_valid) {
+    auto tile_max = [&](int n_valid) {
       float mx = -INFINITY;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
@@ -242,56 +230,65 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
       }
       return mx * a.scale_log2;
     };
-    // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to shared memory, the fp32 sum of the
-    // weights to *sum (H2O only), logits to global (H2O only); returns the largest weight.
-    auto tile_weights = [&](uint32_t s_addr, int pb, int tile_row0, int n_valid, float* sum) {
+    // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
+    // (fp32 for the H2O scores, bf16-rounded for the output) to *sum / *sum_w; logits to global
+    // (H2O only); returns the largest weight.
+    auto tile_weights = [&](int tile_row0, int n_valid, float* sum, float* sum_w) {
       uint32_t pmax = 0u;
-      float acc = 0.f;
+      float acc = 0.f, acc_w = 0.f;
       const bool full = (n_valid == kTM);
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(s_addr + c * 32, v);
+      auto chunk = [&](const uint32_t (&r)[32], int c) {
         if (H2O && live) {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < n_valid) logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = v[j] * a.scale_log2;
+            if (c * 32 + j < n_valid)
+              logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = __uint_as_float(r[j]) * a.scale_log2;
         }
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          float p0 = ex2(fmaf(v[j], a.scale_log2, -m_ref));
-          float p1 = ex2(fmaf(v[j + 1], a.scale_log2, -m_ref));
+          float p0 = ex2(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_ref));
+          float p1 = ex2(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_ref));
           if (!full) {
             if (c * 32 + j >= n_valid) p0 = 0.f;
             if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
           }
           if (H2O) acc += p0 + p1;
-          pk[j / 2] = pack2(p0, p1);
+          // round to bf16 on the integer pipe (nearest, ties up; weights are positive and finite)
+          const uint32_t u0 = (__float_as_uint(p0) + 0x8000u) & 0xffff0000u;
+          const uint32_t u1 = (__float_as_uint(p1) + 0x8000u) & 0xffff0000u;
+          acc_w += __uint_as_float(u0) + __uint_as_float(u1);
+          pk[j / 2] = __byte_perm(u0, u1, 0x7632);
           pmax = max_bf16x2(pmax, pk[j / 2]);
         }
-        // tokens c*32 .. c*32+31 of this row: four 16-byte chunks of P sub-tile (c / 2)
-        if (row < ROWS) {
-          unsigned char* prow = p_s + (pb * 2 + (c >> 1)) * kQBytes + row * 128;
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int chunk = (c & 1) * 4 + q4;
-            *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
-                make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
-          }
-        }
-      }
+        tmem_st16_u32(p_addr + c * 16, pk);  // tokens c*32 .. c*32+31 of this row
+      };
+      // the next chunk's tensor-memory load is in flight while this one is processed
+      uint32_t ra[32], rb[32];
+      tmem_ld32_nowait(s_addr, ra);
+      tmem_wait_ld(ra);
+      tmem_ld32_nowait(s_addr + 32, rb);
+      chunk(ra, 0);
+      tmem_wait_ld(rb);
+      tmem_ld32_nowait(s_addr + 64, ra);
+      chunk(rb, 1);
+      tmem_wait_ld(ra);
+      tmem_ld32_nowait(s_addr + 96, rb);
+      chunk(ra, 2);
+      tmem_wait_ld(rb);
+      chunk(rb, 3);
+      tmem_wait_st();
       *sum = acc;
+      *sum_w = acc_w;
       return fmaxf(__uint_as_float(pmax << 16), __uint_as_float(pmax & 0xffff0000u));
     };
 
     for (int i = 0; ok && i < n_tiles; ++i) {
-      const int buf = i % NSB, pb = i % NSB, st = i % STAGES;
+      const int st = i % STAGES;
       const int tile_row0 = t0 + i * kTM;
       const int n_valid = min(kTM, t1 - tile_row0);
-      const uint32_t s_addr = tmem_base + lane_sel + buf * kTM;
-      ok = mbar_wait(bar_sfull(buf), (i / NSB) & 1, abort_flag);
-      if (ok && i >= NSB) ok = mbar_wait(bar_pfree(pb), ((i / NSB) - 1) & 1, abort_flag);
+      ok = mbar_wait(bar_sfull, i & 1, abort_flag);
+      if (ok && i >= 1) ok = mbar_wait(bar_pfree, (i - 1) & 1, abort_flag);
       if (ok && n_valid < kTM) {
         // rows of the V tile past the unit's last token may hold anything: zero them
         ok = mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag);
@@ -300,53 +297,56 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
 #pragma unroll
           for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0, 0, 0, 0);
         }
+        fence_proxy_async();  // the zeroed rows must be visible to the tensor core
       }
       if (!ok) break;
       tc_fence_after();
       if (warp_live) {
-        if (i == 0) m_ref = tile_max(s_addr, n_valid);
-        float sum;
-        float pmax = tile_weights(s_addr, pb, tile_row0, n_valid, &sum);
+        if (i == 0) m_ref = tile_max(n_valid);
+        float sum, sum_w;
+        float pmax = tile_weights(tile_row0, n_valid, &sum, &sum_w);
         if (__any_sync(0xffffffffu, pmax > kMaxWeight)) {
           // rare: move the reference of the rows that need it; O and the sums (complete up to
           // tile i-1) shrink with it, then the tile is redone.  The whole warp takes part in
           // the TMEM round trip.
-          const float mx2 = tile_max(s_addr, n_valid);
+          const float mx2 = tile_max(n_valid);
           const bool need = pmax > kMaxWeight;
           ok = mbar_wait(bar_odone, (i - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_ref - mx2) : 1.f;
 #pragma unroll 1
-          for (int c = 0; c < 3; ++c) {
+          for (int c = 0; c < 2; ++c) {
             float o[32];
-            tmem_ld32(tmem_o + lane_sel + c * 32, o);
+            tmem_ld32(o_addr + c * 32, o);
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] *= f;
-            tmem_st32(tmem_o + lane_sel + c * 32, o);
+            tmem_st32(o_addr + c * 32, o);
           }
           l_true *= f;
+          l_w *= f;
           if (need) m_ref = mx2;
-          pmax = tile_weights(s_addr, pb, tile_row0, n_valid, &sum);
+          pmax = tile_weights(tile_row0, n_valid, &sum, &sum_w);
         }
         l_true += sum;
+        l_w += sum_w;
       }
-      fence_proxy_async();  // P (and the zeroed V rows) must be visible to the tensor core
       tc_fence_before();
-      mbar_arrive(bar_pready(pb));
-      mbar_arrive(bar_sfree(buf));
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar_pready);
+        mbar_arrive(bar_sfree);
+      }
     }
-    // ---------------- epilogue: O / L -> out (or the split-K partial) ----------------
+    // ---------------- epilogue: O / l -> out (or the split-K partial) ----------------
     if (ok) ok = mbar_wait(bar_odone, (n_tiles - 1) & 1, abort_flag);
     if (ok && warp_live) {
       tc_fence_after();
-      float o[32];
-      tmem_ld32(tmem_o + lane_sel + 2 * 32, o);
-      const float l_w = o[0];  // sum of the bf16 weights that went into O
       const float inv = 1.f / l_w;
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
-        tmem_ld32(tmem_o + lane_sel + c * 32, o);
+        float o[32];
+        tmem_ld32(o_addr + c * 32, o);
         if (!live) continue;
         if (it.n_split == 1) {
 #pragma unroll
@@ -377,11 +377,11 @@ __global__ void __launch_bounds__(192, NSB == 1 ? 2 : 1)
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
 }
 
-template <int STAGES, int ROWS, int NSB, bool H2O>
+template <int STAGES, int ROWS, bool H2O>
 static cudaError_t launch_tc_cfg(const DecodeArgs& a, int n_items, const CUtensorMap& tq, const CUtensorMap& tk,
                                  const CUtensorMap& tv, cudaStream_t s) {
-  constexpr size_t smem = 1024 + (size_t)ROWS * 128 * (1 + 2 * NSB) + (size_t)2 * STAGES * kTileBytes + kOnesBytes + 8 * 16 + 16;
-  auto kern = decode_attn_tc_kernel<STAGES, ROWS, NSB, H2O>;
+  constexpr size_t smem = 1024 + (size_t)ROWS * 128 + (size_t)2 * STAGES * kTileBytes + 8 * 16 + 16;
+  auto kern = decode_attn_tc_kernel<STAGES, ROWS, H2O>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -404,10 +404,10 @@ cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_
     return cudaErrorNotSupported;
   const bool h2o = a.policy == SQ_POLICY_H2O;
   if (rows == 96)
-    return h2o ? launch_tc_cfg<2, 96, 1, true>(a, n_items, tm_q, tm_k, tm_v, s)
-               : launch_tc_cfg<2, 96, 1, false>(a, n_items, tm_q, tm_k, tm_v, s);
-  return h2o ? launch_tc_cfg<3, 128, 2, true>(a, n_items, tm_q, tm_k, tm_v, s)
-             : launch_tc_cfg<3, 128, 2, false>(a, n_items, tm_q, tm_k, tm_v, s);
+    return h2o ? launch_tc_cfg<3, 96, true>(a, n_items, tm_q, tm_k, tm_v, s)
+               : launch_tc_cfg<3, 96, false>(a, n_items, tm_q, tm_k, tm_v, s);
+  return h2o ? launch_tc_cfg<2, 128, true>(a, n_items, tm_q, tm_k, tm_v, s)
+             : launch_tc_cfg<2, 128, false>(a, n_items, tm_q, tm_k, tm_v, s);
 }
 
 }  // namespace sq
