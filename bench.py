@@ -247,6 +247,29 @@ def run_ours(args, w):
     status = job.ctx.status()
     value, ms_max = dist_util.aggregate_throughput(tokens, ms_step, dev)
 
+    # ---- per-layer launches (what a model that computes q layer by layer issues), replayed from
+    # a CUDA graph so that the host's launch cost does not enter ----
+    per_layer = None
+    if not args.no_per_layer:
+        job.prefill(inp)
+        graph = job.capture_decode(inp, per_layer=True)
+        for _ in range(2):
+            job.prefill(inp)
+            graph.replay()
+        torch.cuda.synchronize()
+        n_pl = max(1, min(args.steps, 5))
+        tot = 0.0
+        for _ in range(n_pl):
+            job.prefill(inp)
+            a, b = ev(), ev()
+            a.record()
+            graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        per_layer = {"ms_decode": tot / n_pl, "steps": n_pl}
+        del graph
+
     # ---- end to end: the same pass fed from pinned host memory, outputs copied back ----
     e2e = None
     if not args.no_e2e:
@@ -315,6 +338,11 @@ def run_ours(args, w):
                         "prefill_ms": ms_step - ms_decode},
         "device_status": status,
     }
+    if per_layer is not None:
+        pl_s = per_layer["ms_decode"] * 1e-3
+        line["per_layer_launch"] = {"mode": "one launch per layer per step, CUDA-graph replay",
+                                    "decode_tokens_per_s": tokens / pl_s, "us_per_launch": pl_s * 1e6 / (wr.steps * wr.n_layer),
+                                    "hbm_gbs": alg_bytes * wr.steps / pl_s / 1e9, "hbm_frac": alg_bytes * wr.steps / pl_s / 1e9 / peak}
     print(json.dumps(line), flush=True)
     dist_util.shutdown()
 
@@ -330,6 +358,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-layer", action="store_true", help="skip the per-layer-launch (CUDA graph) measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -89,6 +89,21 @@ class Job:
         self.prefill(inp)
         self.decode(inp)
 
+    def capture_decode(self, inp: ResidentInputs, per_layer: bool):
+        """Captures all decode steps of a pass (one launch per layer if per_layer, else one per
+        step) into a CUDA graph.  Call right after prefill(inp): the kernel arguments, among
+        them each step's token position, are frozen at capture, so the graph replays exactly
+        the steps that follow a prefill of this workload.  The library's host-side step counter
+        advances during capture and not during replay: use replays for timing, and the plain
+        calls when the cache is inspected afterwards."""
+        saved = self.per_layer_decode
+        self.per_layer_decode = per_layer
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.decode(inp)
+        self.per_layer_decode = saved
+        return graph
+
     def kernel_launches_per_pass(self) -> int:
         """Kernels of the library launched by one run(): importance per layer, one allocator,
         prefill kernels per layer, decode kernels per step."""
