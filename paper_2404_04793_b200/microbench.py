@@ -88,6 +88,28 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
                 flops=4 * w.n_q_head * w.head_dim * w.batch * sum(budgets), device_status=ctx.status())
 
 
+def prefill_compress_time(w: synth.Workload, reps=3, device="cuda:0"):
+    """Times sq_prefill_compress of one layer (for H2O: prompt scores on the tensor cores,
+    selection, gather, first victim)."""
+    job = engine.Job(w.replace(steps=1), device)
+    ctx = job.ctx
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets([w.b_init] * w.n_layer)
+    q, k, v = synth.prompt_qkv(w, 0, device, need_q=(w.policy == synth.H2O))
+    ctx.prefill_compress(0, k, v, q)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        ctx.prefill_compress(0, k, v, q)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    flops = 2 * w.batch * w.n_q_head * w.prompt * w.prompt * w.head_dim if w.policy == synth.H2O else 0
+    return dict(workload=w.name, what="prefill_compress, one layer", ms=round(ms, 3),
+                causal_score_flops=flops, tflops=round(flops / ms / 1e9, 1), device_status=ctx.status())
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama2_7b")
@@ -98,7 +120,11 @@ def main():
     ap.add_argument("--steps", type=int, default=12)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
+    ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
     args = ap.parse_args()
+    if args.prefill:
+        print(json.dumps(prefill_compress_time(build_workload(args), args.steps)), flush=True)
+        return
     print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer)), flush=True)
 
 
