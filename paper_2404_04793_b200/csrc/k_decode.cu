@@ -9,7 +9,6 @@
 #include "sq_internal.h"
 #include "sq_select.cuh"
 #include "sq_decode_common.cuh"
-#include "sq_h2o.cuh"
 
 namespace sq {
 
@@ -26,8 +25,6 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
   constexpr int U = 4;           // rows in flight per lane
   __shared__ float sm_o[4][GT][D];
   __shared__ float sm_m[4][GT], sm_l[4][GT];
-  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup];  // H2O: per head, for the score update
-  __shared__ SelScratch sc;
 
   ItemLoc it;
   if (!locate(a, blockIdx.x, -1, it)) return;
@@ -198,8 +195,6 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
         stat[h * kStatStride] = M;
         stat[h * kStatStride + 1] = L;
         stat[h * kStatStride + 2] = L;
-        s_M[h] = M;
-        s_invL[h] = 1.f / L;
       }
     }
     __syncthreads();
@@ -219,10 +214,6 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
       if (h2o) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
     }
   }
-  if (h2o && it.n_split == 1) {
-    __syncthreads();  // logits, the new token's tables and s_M / s_invL are in place
-    h2o_update_unit(a, ldp, unit, s_M, s_invL, sc);
-  }
 }
 
 // One CTA per (layer, unit): merges the split-K partials into the output and, for H2O, adds
@@ -239,8 +230,8 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
   ItemLoc it;
   if (!locate(a, 0, layer, it)) return;
   const int tid = threadIdx.x, D = a.head_dim, G = a.group, ns = it.n_split;
-  if (ns == 1) return;  // an unsplit unit is finished (output, scores, victim) by its attention CTA
   const LayerDesc* ldp = a.layers + layer;
+  const int b = ldp->b, cap = ldp->cap;
   const size_t item0 = (size_t)it.base + (size_t)unit * ns;
   const float* stat = a.part_stat + item0 * G * kStatStride;
   for (int h = tid; h < G; h += kSelThreads) {
@@ -274,7 +265,34 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
     }
   }
   if (a.policy != SQ_POLICY_H2O) return;
-  h2o_update_unit(a, ldp, unit, s_M, s_invL, sc);
+  const int len = min(a.n_tok + 1, b);
+  const bool full = (len == b);
+  const int thr = a.n_tok + 1 - ldp->b_recent;  // next step: positions <= thr are outside the recent window
+  const int* pos = reinterpret_cast<const int*>(a.pool + ldp->pos_off) + (size_t)unit * cap;
+  float* acc = reinterpret_cast<float*>(a.pool + ldp->acc_off) + (size_t)unit * cap;
+  const float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  unsigned long long best = ~0ull;
+  int best_slot = -1;
+  for (int slot = tid; slot < len; slot += kSelThreads) {
+    float gain = 0.f;
+    for (int h = 0; h < G; ++h) gain += exp2f(logit[(size_t)slot * G + h] - s_M[h]) * s_invL[h];
+    const float v = acc[slot] + gain;
+    acc[slot] = v;
+    if (full) {
+      const int p = pos[slot];
+      if (p <= thr) {
+        const unsigned long long r = victim_rank(v, p);
+        if (r < best) {
+          best = r;
+          best_slot = slot;
+        }
+      }
+    }
+  }
+  if (full) {
+    best_slot = block_argmin(sc, best, best_slot);
+    if (tid == 0) reinterpret_cast<int*>(a.pool + ldp->victim_off)[unit] = best_slot;
+  }
 }
 
 template <typename T, int D>

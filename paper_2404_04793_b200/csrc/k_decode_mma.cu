@@ -9,7 +9,6 @@
 // XOR-swizzled rows so ldmatrix is bank-conflict free).  Warps split the tile's tokens (WN)
 // and, for very wide groups, the head tiles (WM); partial results merge through shared memory.
 #include "sq_decode_common.cuh"
-#include "sq_h2o.cuh"
 #include "sq_device.cuh"
 #include "sq_internal.h"
 
@@ -77,8 +76,6 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
   static_assert(kTile / WN == 16, "each warp owns 16 tokens of a tile");
   using bf16 = __nv_bfloat16;
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup];  // H2O: per head, for the score update
-  __shared__ SelScratch sc;
   unsigned char* q_s = smem;
   unsigned char* k_s = smem + QROWS * D * 2;
   unsigned char* v_s = k_s + STAGES * TILE_BYTES;
@@ -342,7 +339,7 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
     }
     __syncthreads();
   }
-  if (wn == 0) {
+  if (wn != 0) return;
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -365,15 +362,8 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
         stat[h * kStatStride] = m_run[mt][hf];
         stat[h * kStatStride + 1] = l_true[mt][hf];
         stat[h * kStatStride + 2] = l_w[mt][hf];
-        s_M[h] = m_run[mt][hf];
-        s_invL[h] = 1.f / l_true[mt][hf];
       }
     }
-  }
-  if (h2o && it.n_split == 1) {
-    __syncthreads();  // logits and s_M / s_invL are in place
-    h2o_update_unit(a, ldp, unit, s_M, s_invL, sc);
-  }
 }
 
 template <int D, int MT, int WM, int WN, int STAGES>

@@ -18,7 +18,6 @@
 // tcgen05.ld/st, the tile redone): every weight stays finite and the result is that of the
 // exact softmax.  Every barrier wait is bounded.
 #include "sq_decode_common.cuh"
-#include "sq_h2o.cuh"
 #include "sq_internal.h"
 #include "sq_tc.cuh"
 
@@ -54,8 +53,6 @@ __global__ void __launch_bounds__(192, 2)
                           const __grid_constant__ CUtensorMap tm_v, DecodeArgs a) {
   constexpr int kQBytes = ROWS * 128;
   extern __shared__ unsigned char smem_raw[];
-  __shared__ float s_M[H2O ? kMaxGroup : 1], s_invL[H2O ? kMaxGroup : 1];  // per head, for the score update
-  __shared__ SelScratch sc;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   // The first MMA addresses 128 rows of Q; with ROWS = 96 rows 96..127 alias the K stage that
   // follows (rows are independent, those accumulator rows are never read).
@@ -368,10 +365,6 @@ __global__ void __launch_bounds__(192, 2)
         stat[row * kStatStride] = m_ref;
         stat[row * kStatStride + 1] = H2O ? l_true : l_w;
         stat[row * kStatStride + 2] = l_w;
-        if (H2O) {
-          s_M[row] = m_ref;
-          s_invL[row] = 1.f / l_true;
-        }
       }
     }
   }
@@ -382,10 +375,6 @@ __global__ void __launch_bounds__(192, 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
-  if (H2O && it.n_split == 1 && !*abort_flag) {
-    __syncthreads();
-    h2o_update_unit(a, ldp, unit, s_M, s_invL, sc);
-  }
 }
 
 template <int STAGES, int ROWS, bool H2O>

@@ -474,7 +474,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.split_tokens = split;
     a.policy = cfg.policy;
     a.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg.head_dim));
-    const bool combine = any_split;  // unsplit units are finished inside the attention kernel
+    const bool combine = any_split || cfg.policy == SQ_POLICY_H2O;
     SQ_CUDA(c, launch_decode(a, cfg.dtype, (int)n_items, combine, c->pool_bytes,
                              (size_t)(e - s) * c->batch * cfg.n_q_head, st));
     for (int l = s; l < e; ++l) c->n_tok[l] += 1;

@@ -108,8 +108,8 @@ __device__ __forceinline__ int block_argmin(SelScratch& sc, unsigned long long c
   __syncthreads();
   unsigned long long bc = sc.best[0];
   int bs = sc.best_slot[0];
-  const int n_warp = blockDim.x >> 5;  // blocks of up to kSelThreads threads
-  for (int w = 1; w < n_warp; ++w) {
+#pragma unroll
+  for (int w = 1; w < kSelThreads / 32; ++w) {
     if (sc.best[w] < bc) {
       bc = sc.best[w];
       bs = sc.best_slot[w];
