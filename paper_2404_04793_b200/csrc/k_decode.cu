@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
 template <typename T>
 __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
   __shared__ SelScratch sc;
-  __shared__ float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
+  __shared__ __align__(16) float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
   const int n_layers = a.layer_end - a.layer_begin;
   const int layer = a.layer_begin + blockIdx.x / a.n_unit;
   const int unit = blockIdx.x % a.n_unit;
@@ -273,15 +273,55 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
   const float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
   unsigned long long best = ~0ull;
   int best_slot = -1;
-  for (int slot = tid; slot < len; slot += kSelThreads) {
-    float gain = 0.f;
-    for (int h = 0; h < G; ++h) gain += exp2f(logit[(size_t)slot * G + h] - s_M[h]) * s_invL[h];
-    const float v = acc[slot] + gain;
-    acc[slot] = v;
-    if (full) {
-      const int p = pos[slot];
-      if (p <= thr) {
-        const unsigned long long r = victim_rank(v, p);
+  // four slots per thread in flight: their logits, score and position loads are independent
+  constexpr int kIl = 4;
+  for (int s0 = tid; s0 < len; s0 += kIl * kSelThreads) {
+    float gain[kIl], old[kIl];
+    int p[kIl];
+#pragma unroll
+    for (int u = 0; u < kIl; ++u) {
+      const int slot = s0 + u * kSelThreads;
+      gain[u] = 0.f;
+      old[u] = 0.f;
+      p[u] = 0x7fffffff;
+      if (slot < len) {
+        old[u] = acc[slot];
+        if (full) p[u] = pos[slot];
+      }
+    }
+    if ((G & 3) == 0) {
+      for (int h = 0; h < G; h += 4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(s_M + h), i4 = *reinterpret_cast<const float4*>(s_invL + h);
+#pragma unroll
+        for (int u = 0; u < kIl; ++u) {
+          const int slot = s0 + u * kSelThreads;
+          if (slot < len) {
+            const float4 l4 = *reinterpret_cast<const float4*>(logit + (size_t)slot * G + h);
+            gain[u] += exp2f(l4.x - m4.x) * i4.x;
+            gain[u] += exp2f(l4.y - m4.y) * i4.y;
+            gain[u] += exp2f(l4.z - m4.z) * i4.z;
+            gain[u] += exp2f(l4.w - m4.w) * i4.w;
+          }
+        }
+      }
+    } else {
+      for (int h = 0; h < G; ++h) {
+        const float mh = s_M[h], ih = s_invL[h];
+#pragma unroll
+        for (int u = 0; u < kIl; ++u) {
+          const int slot = s0 + u * kSelThreads;
+          if (slot < len) gain[u] += exp2f(logit[(size_t)slot * G + h] - mh) * ih;
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kIl; ++u) {
+      const int slot = s0 + u * kSelThreads;
+      if (slot >= len) continue;
+      const float v = old[u] + gain[u];
+      acc[slot] = v;
+      if (full && p[u] <= thr) {
+        const unsigned long long r = victim_rank(v, p[u]);
         if (r < best) {
           best = r;
           best_slot = slot;
