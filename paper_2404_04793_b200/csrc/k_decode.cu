@@ -305,13 +305,14 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
         }
       }
     } else {
-      for (int h = 0; h < G; ++h) {
-        const float mh = s_M[h], ih = s_invL[h];
-#pragma unroll
-        for (int u = 0; u < kIl; ++u) {
-          const int slot = s0 + u * kSelThreads;
-          if (slot < len) gain[u] += exp2f(logit[(size_t)slot * G + h] - mh) * ih;
-        }
+      // odd group sizes: one slot at a time, so a slot's G consecutive logits stay in L1
+#pragma unroll 1
+      for (int u = 0; u < kIl; ++u) {
+        const int slot = s0 + u * kSelThreads;
+        if (slot >= len) continue;
+        float g1 = 0.f;
+        for (int h = 0; h < G; ++h) g1 += exp2f(logit[(size_t)slot * G + h] - s_M[h]) * s_invL[h];
+        gain[u] = g1;
       }
     }
 #pragma unroll
