@@ -121,7 +121,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
+    ap.add_argument("--sweep-falcon", action="store_true",
+                    help="decode-step time over the Falcon-7B-shaped grid: batch x prompt x budget x policy")
     args = ap.parse_args()
+    if args.sweep_falcon:
+        for policy in ("sliding_window", "streaming_llm", "h2o"):
+            for batch in (1, 8, 32, 128, 224):
+                for prompt in (512, 2048, 8192, 16384):
+                    for pct in (10.0, 20.0, 30.0, 50.0):
+                        w = synth.falcon_7b(batch, prompt, pct, POLICIES[policy])
+                        r = decode_step_time(w, args.steps, args.warmup)
+                        r.update(policy=policy, batch=batch, prompt=prompt, budget_pct=pct)
+                        print(json.dumps(r), flush=True)
+                        torch.cuda.empty_cache()
+        return
     if args.prefill:
         print(json.dumps(prefill_compress_time(build_workload(args), args.steps)), flush=True)
         return
