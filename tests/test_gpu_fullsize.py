@@ -1,4 +1,4 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (one fused
+"""Parity at the full sizes of the paper-shaped workloads, in the launch configuration bench.py times (one fused
 decode launch per step over all layers): sampled (layer, sequence, KV head) units are
 followed by the oracle through every step.  Units are independent, so a sample that always
 holds the first and last unit and every layer of one sequence covers the layout arithmetic."""

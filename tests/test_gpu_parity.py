@@ -393,3 +393,28 @@ def test_call_order_and_argument_errors():
     with pytest.raises(B.SqError) as e:
         c2.set_budgets([30, 4, 30])              # a budget that leaves no room beside the sinks
     assert e.value.code == B.SQ_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------- launch forms agree
+def test_graph_replay_and_per_layer_calls_match_fused_launch():
+    """The same decode steps issued as one launch per step, as one launch per layer, and as a
+    CUDA-graph replay of the per-layer launches give identical bits."""
+    from paper_2404_04793_b200 import engine
+    w = small("forms", 31, policy=synth.STREAMING_LLM, dtype=torch.bfloat16, head_dim=128, n_q_head=8, n_kv_head=2,
+              n_layer=4, steps=5)
+    inp = engine.ResidentInputs(w, DEV)
+    outs = []
+    for mode in ("fused", "per_layer", "graph"):
+        job = engine.Job(w, DEV, per_layer_decode=(mode == "per_layer"))
+        job.prefill(inp)
+        if mode == "graph":
+            graph = job.capture_decode(inp, per_layer=True)
+            job.prefill(inp)
+            graph.replay()
+        else:
+            job.decode(inp)
+        torch.cuda.synchronize()
+        assert job.ctx.status() == 0
+        outs.append(job.out.clone())
+    assert torch.equal(outs[0], outs[1])
+    assert torch.equal(outs[0], outs[2])
