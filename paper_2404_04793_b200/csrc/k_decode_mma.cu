@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
     }
     __syncthreads();
   }
-  if (wn != 0) return;
+  if (wn == 0) {
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -364,6 +364,8 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
         stat[h * kStatStride + 2] = l_w[mt][hf];
       }
     }
+  }
+  if (!h2o && it.n_split > 1) merge_if_last<bf16>(a, it, unit);
 }
 
 template <int D, int MT, int WM, int WN, int STAGES>

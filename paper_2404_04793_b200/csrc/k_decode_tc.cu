@@ -375,6 +375,7 @@ __global__ void __launch_bounds__(192, 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
+  if (!H2O && it.n_split > 1) merge_if_last<bf16>(a, it, unit);
 }
 
 template <int STAGES, int ROWS, bool H2O>

@@ -20,7 +20,7 @@ inline int elem_bytes(int dtype) { return dtype == SQ_F32 ? 4 : 2; }
 constexpr int kMaxImportanceCtas = 4096;
 
 struct WsLayout {
-  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, layers, order;
+  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order;
   size_t part_stat, part_o, logits, acc_prompt, lse2, total;
   size_t items_cap, logits_floats;
 };
@@ -113,6 +113,7 @@ WsLayout ws_layout(const sq_config& c, int64_t b_init) {
   w.budget = take(4 * L);
   w.is_g3 = take(L);
   w.status = take(4);
+  w.tickets = take(4 * L * U);
   w.layers = take(sizeof(LayerDesc) * L);
   w.order = take(4 * L);
   w.items_cap = (size_t)kTargetItems + U * L;
@@ -438,8 +439,9 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     long long total = 0;
     for (int l = s; l < e; ++l) total += (long long)U * std::min(n_tok + 1, c->hs->layers[l].b);
     int split = 1 << 30;
+    const bool wide = cfg.dtype == SQ_BF16 && cfg.head_dim == 64 && G > 32;  // 128-token tiles
     if ((long long)U * (e - s) < kTargetItems / 2)
-      split = (int)std::max<long long>(kMinSplitTokens, (total + kTargetItems - 1) / kTargetItems);
+      split = (int)std::max<long long>(wide ? 256 : kMinSplitTokens, (total + kTargetItems - 1) / kTargetItems);
     long long n_items = 0;
     bool any_split = false;
     for (int l = s; l < e; ++l) {
@@ -461,6 +463,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.v_new = static_cast<const char*>(v_new) + (size_t)(s - layer_begin) * kv_layer;
     a.out = static_cast<char*>(out) + (size_t)(s - layer_begin) * q_layer;
     a.status = ws_ptr<int>(c, c->wl.status);
+    a.tickets = ws_ptr<int>(c, c->wl.tickets);
     a.n_layer_total = cfg.n_layer;
     a.layer_begin = s;
     a.layer_end = e;
@@ -474,7 +477,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.split_tokens = split;
     a.policy = cfg.policy;
     a.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg.head_dim));
-    const bool combine = any_split || cfg.policy == SQ_POLICY_H2O;
+    const bool combine = cfg.policy == SQ_POLICY_H2O;  // other policies merge split-K pieces in the last piece
     SQ_CUDA(c, launch_decode(a, cfg.dtype, (int)n_items, combine, c->pool_bytes,
                              (size_t)(e - s) * c->batch * cfg.n_q_head, st));
     for (int l = s; l < e; ++l) c->n_tok[l] += 1;

@@ -1,5 +1,7 @@
 // Work-item numbering shared by the decode kernels.
 #pragma once
+#include <cuda_bf16.h>
+
 #include "sq_internal.h"
 
 namespace sq {
@@ -54,6 +56,59 @@ __device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_la
     running += __shfl_sync(kFull, incl, 31);
   }
   return false;
+}
+
+
+// Split-K merge without a second launch (policies without scores): every piece of a unit
+// bumps the unit's ticket after its partials are written; the piece that arrives last reads
+// all of them back (in piece order, so the result does not depend on who merges), writes the
+// output and resets the ticket.  No piece ever waits for another.
+template <typename T>
+__device__ __forceinline__ void merge_if_last(const DecodeArgs& a, const ItemLoc& it, int unit) {
+  __shared__ int s_last;
+  __shared__ float s_mM[kMaxGroup], s_mInv[kMaxGroup];
+  const int tid = threadIdx.x, nt = blockDim.x, G = a.group, D = a.head_dim, ns = it.n_split;
+  int* ticket = a.tickets + (size_t)it.layer * a.n_unit + unit;
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    s_last = (atomicAdd(ticket, 1) == ns - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (tid == 0) *ticket = 0;
+  const size_t item0 = (size_t)it.base + (size_t)unit * ns;
+  const float* stat = a.part_stat + item0 * G * kStatStride;
+  for (int h = tid; h < G; h += nt) {
+    float M = -INFINITY;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(stat + ((size_t)s * G + h) * kStatStride));
+    float Lw = 0.f;
+    for (int s = 0; s < ns; ++s) {
+      const float* st = stat + ((size_t)s * G + h) * kStatStride;
+      const float ms = __ldcg(st);
+      Lw += __ldcg(st + 2) * ((ms > -INFINITY) ? exp2f(ms - M) : 0.f);
+    }
+    s_mM[h] = M;
+    s_mInv[h] = 1.f / Lw;
+  }
+  __syncthreads();
+  const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
+  const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
+  T* ob = reinterpret_cast<T*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * D;
+  const float* po = a.part_o + item0 * G * D;
+  for (int idx = tid; idx < G * D; idx += nt) {
+    const int h = idx / D;
+    float O = 0.f;
+    for (int s = 0; s < ns; ++s) {
+      const float ms = __ldcg(stat + ((size_t)s * G + h) * kStatStride);
+      O += __ldcg(po + (size_t)s * G * D + idx) * ((ms > -INFINITY) ? exp2f(ms - s_mM[h]) : 0.f);
+    }
+    if (sizeof(T) == 2)
+      reinterpret_cast<__nv_bfloat16*>(ob)[idx] = __float2bfloat16_rn(O * s_mInv[h]);
+    else
+      reinterpret_cast<float*>(ob)[idx] = O * s_mInv[h];
+  }
 }
 
 }  // namespace sq

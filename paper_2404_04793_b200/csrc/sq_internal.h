@@ -10,7 +10,7 @@ namespace sq {
 
 constexpr int kMaxLayers = 256;
 constexpr int kMaxGroup = 128;          // query heads per KV head
-constexpr int kMinSplitTokens = 256;    // a split-K piece is never shorter than this
+constexpr int kMinSplitTokens = 64;     // a split-K piece is never shorter than this (256 for the tcgen05 kernel)
 constexpr int kTargetItems = 148 * 16;  // decode CTAs wanted per launch before split-K stops
 
 // Per-layer cache geometry, resident in device memory once the budgets are known.
@@ -81,6 +81,7 @@ struct DecodeArgs {
   const void* v_new;
   void* out;
   int* status;
+  int* tickets;  // [n_layer_total][n_unit] arrival counters of the split-K pieces, zero between launches
   int n_layer_total, layer_begin, layer_end;
   int n_tok;  // tokens seen before this step == position of the new token
   int batch, n_q_head, n_kv_head, head_dim, group;
