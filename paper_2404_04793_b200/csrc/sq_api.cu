@@ -439,9 +439,15 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     long long total = 0;
     for (int l = s; l < e; ++l) total += (long long)U * std::min(n_tok + 1, c->hs->layers[l].b);
     int split = 1 << 30;
-    const bool wide = cfg.dtype == SQ_BF16 && cfg.head_dim == 64 && G > 32;  // 128-token tiles
-    if ((long long)U * (e - s) < kTargetItems / 2)
-      split = (int)std::max<long long>(wide ? 256 : kMinSplitTokens, (total + kTargetItems - 1) / kTargetItems);
+    // Split-K only when the units alone cannot fill the GPU.  How many CTAs that takes depends on
+    // the kernel: the fp32-pipe kernel is light (7 CTAs per SM), the tensor-core kernels carry
+    // a shared-memory pipeline (2 per SM) and pay a fixed set-up per CTA, so they want few,
+    // long pieces.
+    const bool tensor = cfg.dtype == SQ_BF16 && G > 1;
+    const bool wide = tensor && cfg.head_dim == 64 && G > 32;  // 128-token tiles
+    const long long target = tensor ? 6LL * c->n_sm : 8LL * c->n_sm;
+    if ((long long)U * (e - s) < target / 2)
+      split = (int)std::max<long long>(tensor ? 256 : kMinSplitTokens, (total + target - 1) / target);
     long long n_items = 0;
     bool any_split = false;
     for (int l = s; l < e; ++l) {
