@@ -232,9 +232,8 @@ __global__ void __launch_bounds__(192, 2)
     };
     // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
     // (fp32 for the H2O scores, bf16-rounded for the output) to *sum / *sum_w; logits to global
-    // (H2O only); returns the largest weight.
+    // (H2O only); returns an upper bound of the largest weight.
     auto tile_weights = [&](int tile_row0, int n_valid, float* sum, float* sum_w) {
-      uint32_t pmax = 0u;
       float acc = 0.f, acc_w = 0.f;
       const bool full = (n_valid == kTM);
       auto chunk = [&](const uint32_t (&r)[32], int c) {
@@ -254,12 +253,9 @@ __global__ void __launch_bounds__(192, 2)
             if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
           }
           if (H2O) acc += p0 + p1;
-          // round to bf16 on the integer pipe (nearest, ties up; weights are positive and finite)
-          const uint32_t u0 = (__float_as_uint(p0) + 0x8000u) & 0xffff0000u;
-          const uint32_t u1 = (__float_as_uint(p1) + 0x8000u) & 0xffff0000u;
-          acc_w += __uint_as_float(u0) + __uint_as_float(u1);
-          pk[j / 2] = __byte_perm(u0, u1, 0x7632);
-          pmax = max_bf16x2(pmax, pk[j / 2]);
+          const uint32_t u = pack2(p0, p1);  // round to nearest bf16, p0 in the low half
+          acc_w += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
+          pk[j / 2] = u;
         }
         tmem_st16_u32(p_addr + c * 16, pk);  // tokens c*32 .. c*32+31 of this row
       };
@@ -280,7 +276,7 @@ __global__ void __launch_bounds__(192, 2)
       tmem_wait_st();
       *sum = acc;
       *sum_w = acc_w;
-      return fmaxf(__uint_as_float(pmax << 16), __uint_as_float(pmax & 0xffff0000u));
+      return acc_w;  // the tile's weight sum bounds its largest weight
     };
 
     for (int i = 0; ok && i < n_tiles; ++i) {
