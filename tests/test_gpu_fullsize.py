@@ -88,3 +88,8 @@ def test_falcon_7b_mqa_cells():
     for policy, batch, prompt, pct in [(synth.SLIDING_WINDOW, 32, 2048, 20.0), (synth.STREAMING_LLM, 8, 8192, 10.0),
                                        (synth.H2O, 2, 2048, 30.0)]:
         _follow(synth.falcon_7b(batch, prompt, pct, policy), n_units=34, steps=4)
+
+
+def test_falcon_7b_largest_cell_sampled():
+    # the largest cell of the sweep: batch 224, prompt 16384, budget 50 % (15 GB of K/V per step)
+    _follow(synth.falcon_7b(224, 16384, 50.0, synth.SLIDING_WINDOW), n_units=36, steps=2)
