@@ -18,7 +18,7 @@ namespace sq {
 // and of their output accumulators in fp32; logits are reduced over the LPR lanes by
 // shuffles, and the softmax runs online in the log2 domain over batches of U rows.
 template <typename T, int D, int GT>
-__global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(128, GT == 1 ? 7 : 1) decode_attn_kernel(DecodeArgs a) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;   // lanes per row
   constexpr int RPW = 32 / LPR;  // rows per warp per load

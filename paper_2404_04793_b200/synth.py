@@ -122,15 +122,16 @@ def cos_targets(n_layer: int):
     return c
 
 
-def hidden_pair(w: Workload, layer: int, device="cpu", batch=None, n_tok=None):
+def hidden_pair(w: Workload, layer: int, device="cpu", batch=None, n_tok=None, chunk=0):
     """(hidden_in, hidden_out), each [B, P, hidden]: the state before and after
     self-attention.  hidden_out = hidden_in + alpha_l * noise with alpha_l set
-    from the layer's target similarity."""
+    from the layer's target similarity.  Large batches can be drawn in pieces:
+    `batch` sequences per call, `chunk` numbering the pieces."""
     B = w.batch if batch is None else batch
     P = w.prompt if n_tok is None else n_tok
     c = cos_targets(w.n_layer)[layer]
     alpha = math.sqrt(1.0 / (c * c) - 1.0)
-    g = _gen(w, 0, layer, device=device)
+    g = _gen(w, 0, layer, chunk, device=device)
     a = torch.randn(B, P, w.hidden, generator=g, device=device, dtype=torch.float32)
     n = torch.randn(B, P, w.hidden, generator=g, device=device, dtype=torch.float32)
     b = a + alpha * n
