@@ -110,6 +110,68 @@ def prefill_compress_time(w: synth.Workload, reps=3, device="cuda:0"):
                 causal_score_flops=flops, tflops=round(flops / ms / 1e9, 1), device_status=ctx.status())
 
 
+def generation_throughput(w: synth.Workload, device="cuda:0"):
+    """Decode tokens/s of the attention + eviction path over a whole generation: cache filled
+    from a prompt of w.prompt tokens, then w.steps fused decode steps, all timed together."""
+    job = engine.Job(w, device)
+    ctx = job.ctx
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    for l in range(w.n_layer):
+        a, b = synth.hidden_pair(w, l, device, batch=1, n_tok=min(256, w.prompt))
+        ctx.layer_importance(l, a, b)
+    ctx.allocate_budgets(w.b_init, w.p)
+    budgets, _ = ctx.get_budgets()
+    g = torch.Generator(device=device).manual_seed(1)
+    shape_kv = (w.batch, w.n_kv_head, w.prompt, w.head_dim)
+    k = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    v = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    acc = torch.rand(w.batch, w.n_kv_head, w.prompt, generator=g, device=device) if w.policy == synth.H2O else None
+    q = torch.randn(w.n_layer, w.batch, w.n_q_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    kn = torch.randn(w.n_layer, w.batch, w.n_kv_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    vn = torch.randn(w.n_layer, w.batch, w.n_kv_head, w.head_dim, generator=g, device=device).to(w.dtype)
+    out = torch.empty_like(q)
+
+    def one_generation():
+        for l in range(w.n_layer):
+            ctx.prefill_compress(l, k, v, None, acc)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(w.steps):
+            ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    one_generation()
+    ms = one_generation()
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    cache_gb = w.batch * w.n_kv_head * sum(min(w.prompt + w.steps, b) for b in budgets) * 2 * w.head_dim * e / 1e9
+    return dict(workload=w.name, batch=w.batch, budget_pct=w.budget_pct, p=w.p, ms_total=round(ms, 2),
+                tokens_per_s=round(w.batch * w.steps / ms * 1e3), final_cache_GB=round(cache_gb, 2),
+                device_status=ctx.status())
+
+
+def compare_budgets():
+    """Full cache vs a sequence-wise policy alone vs the layer-wise reallocation on the same
+    kernels, on the shapes of the paper's throughput table (attention path only, no weights)."""
+    rows = []
+    shapes = [("mistral_7b", 512, 1024, synth.SLIDING_WINDOW, (1, 32, 64, 128, 224), 30.0, 20.0, 0.35),
+              ("llama2_70b", 256, 512, synth.STREAMING_LLM, (1, 8, 16, 32, 64), 40.0, 30.0, 0.3)]
+    for name, P, T, policy, batches, pct_alone, pct_squeeze, p in shapes:
+        base = synth.WORKLOADS[name]().replace(prompt=P, steps=T, policy=policy)
+        full_pct = 100.0 * (P + T) / P + 1.0
+        for batch in batches:
+            for label, pct, pp in (("full cache", full_pct, 1.0), ("sequence-wise alone", pct_alone, 1.0),
+                                   ("layer-wise budgets", pct_squeeze, p)):
+                w = base.replace(batch=batch, budget_pct=pct, p=pp, name=f"{name}_{label.replace(' ', '_')}")
+                r = generation_throughput(w)
+                r.update(shape=name, variant=label, prompt=P, gen=T)
+                rows.append(r)
+                print(json.dumps(r), flush=True)
+                torch.cuda.empty_cache()
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama2_7b")
@@ -121,9 +183,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
+    ap.add_argument("--compare-budgets", action="store_true",
+                    help="generation throughput: full cache vs sequence-wise policy alone vs layer-wise budgets")
     ap.add_argument("--sweep-falcon", action="store_true",
                     help="decode-step time over the Falcon-7B-shaped grid: batch x prompt x budget x policy")
     args = ap.parse_args()
+    if args.compare_budgets:
+        compare_budgets()
+        return
     if args.sweep_falcon:
         for policy in ("sliding_window", "streaming_llm", "h2o"):
             for batch in (1, 8, 32, 128, 224):
