@@ -366,8 +366,14 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   bool done = false;
   if (dtype == SQ_BF16 && ovr == 0 && a.group > 32) {
     cudaError_t e = launch_decode_attn_tc(a, n_items, pool_bytes, q_rows, s);
-    if (e == cudaSuccess) done = true;
-    else if (e != cudaErrorNotSupported) return e;
+    if (e == cudaSuccess) {
+      // H2O: the attention kernel left the row log-sum-exps; the scores and the next victim come
+      // from a second pass over K instead of logits carried through memory
+      if (a.policy == SQ_POLICY_H2O) return launch_h2o_gain_tc(a, n_items, pool_bytes, q_rows, s);
+      done = true;
+    } else if (e != cudaErrorNotSupported) {
+      return e;
+    }
   }
   if (!done && dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
     cudaError_t e = launch_decode_attn_mma(a, n_items, s);

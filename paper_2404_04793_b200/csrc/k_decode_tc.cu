@@ -95,7 +95,8 @@ __global__ void __launch_bounds__(192, 2)
   const bf16* kn = reinterpret_cast<const bf16*>(a.k_new) + (tok * a.n_kv_head + kvh) * kD;
   const bf16* vn = reinterpret_cast<const bf16*>(a.v_new) + (tok * a.n_kv_head + kvh) * kD;
   bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
-  float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  // H2O: the unit's row log-sum-exps (log2 domain), read by the score-update pass that follows
+  float* lse = a.logits + ldp->logit_off + (size_t)unit * cap * G;
   float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
   float* po = a.part_o + (size_t)blockIdx.x * G * kD;
   // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q
@@ -231,18 +232,12 @@ __global__ void __launch_bounds__(192, 2)
       return mx * a.scale_log2;
     };
     // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
-    // (fp32 for the H2O scores, bf16-rounded for the output) to *sum / *sum_w; logits to global
-    // (H2O only); returns an upper bound of the largest weight.
-    auto tile_weights = [&](int tile_row0, int n_valid, float* sum, float* sum_w) {
+    // (fp32 for the H2O normaliser, bf16-rounded for the output) to *sum / *sum_w; returns an
+    // upper bound of the largest weight.
+    auto tile_weights = [&](int n_valid, float* sum, float* sum_w) {
       float acc = 0.f, acc_w = 0.f;
       const bool full = (n_valid == kTM);
       auto chunk = [&](const uint32_t (&r)[32], int c) {
-        if (H2O && live) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < n_valid)
-              logit[(size_t)(tile_row0 + c * 32 + j) * G + row] = __uint_as_float(r[j]) * a.scale_log2;
-        }
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
@@ -300,7 +295,7 @@ __global__ void __launch_bounds__(192, 2)
       if (warp_live) {
         if (i == 0) m_ref = tile_max(n_valid);
         float sum, sum_w;
-        float pmax = tile_weights(tile_row0, n_valid, &sum, &sum_w);
+        float pmax = tile_weights(n_valid, &sum, &sum_w);
         if (__any_sync(0xffffffffu, pmax > kMaxWeight)) {
           // rare: move the reference of the rows that need it; O and the sums (complete up to
           // tile i-1) shrink with it, then the tile is redone.  The whole warp takes part in
@@ -322,7 +317,7 @@ __global__ void __launch_bounds__(192, 2)
           l_true *= f;
           l_w *= f;
           if (need) m_ref = mx2;
-          pmax = tile_weights(tile_row0, n_valid, &sum, &sum_w);
+          pmax = tile_weights(n_valid, &sum, &sum_w);
         }
         l_true += sum;
         l_w += sum_w;
@@ -361,6 +356,7 @@ __global__ void __launch_bounds__(192, 2)
         stat[row * kStatStride] = m_ref;
         stat[row * kStatStride + 1] = H2O ? l_true : l_w;
         stat[row * kStatStride + 2] = l_w;
+        if (H2O && it.n_split == 1) lse[row] = m_ref + log2f(l_true);
       }
     }
   }
@@ -371,7 +367,7 @@ __global__ void __launch_bounds__(192, 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
-  if (!H2O && it.n_split > 1) merge_if_last<bf16>(a, it, unit);
+  if (it.n_split > 1) merge_if_last<bf16>(a, it, unit, H2O ? lse : nullptr);
 }
 
 template <int STAGES, int ROWS, bool H2O>

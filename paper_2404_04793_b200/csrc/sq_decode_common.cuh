@@ -62,9 +62,11 @@ __device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_la
 // Split-K merge without a second launch (policies without scores): every piece of a unit
 // bumps the unit's ticket after its partials are written; the piece that arrives last reads
 // all of them back (in piece order, so the result does not depend on who merges), writes the
-// output and resets the ticket.  No piece ever waits for another.
+// output and resets the ticket.  No piece ever waits for another.  With lse_out set, the merged
+// log-sum-exp (log2 domain, from the unrounded weight sums) of every head is stored there too.
 template <typename T>
-__device__ __forceinline__ void merge_if_last(const DecodeArgs& a, const ItemLoc& it, int unit) {
+__device__ __forceinline__ void merge_if_last(const DecodeArgs& a, const ItemLoc& it, int unit,
+                                              float* lse_out = nullptr) {
   __shared__ int s_last;
   __shared__ float s_mM[kMaxGroup], s_mInv[kMaxGroup];
   const int tid = threadIdx.x, nt = blockDim.x, G = a.group, D = a.head_dim, ns = it.n_split;
@@ -83,14 +85,17 @@ __device__ __forceinline__ void merge_if_last(const DecodeArgs& a, const ItemLoc
   for (int h = tid; h < G; h += nt) {
     float M = -INFINITY;
     for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(stat + ((size_t)s * G + h) * kStatStride));
-    float Lw = 0.f;
+    float Lw = 0.f, Lt = 0.f;
     for (int s = 0; s < ns; ++s) {
       const float* st = stat + ((size_t)s * G + h) * kStatStride;
       const float ms = __ldcg(st);
-      Lw += __ldcg(st + 2) * ((ms > -INFINITY) ? exp2f(ms - M) : 0.f);
+      const float f = (ms > -INFINITY) ? exp2f(ms - M) : 0.f;
+      Lw += __ldcg(st + 2) * f;
+      if (lse_out) Lt += __ldcg(st + 1) * f;
     }
     s_mM[h] = M;
     s_mInv[h] = 1.f / Lw;
+    if (lse_out) lse_out[h] = M + log2f(Lt);
   }
   __syncthreads();
   const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
