@@ -10,8 +10,12 @@
 // p = exp2(s*scale - lse_h) are summed over the heads in registers (no shuffles, no atomics,
 // head order fixed: deterministic), and the score read-modify-write is one coalesced access.
 //   warp 0      TMA: Q once, K tiles into a ring of stages (128-byte swizzle, no multicast)
-//   warp 1      MMA issue, two accumulator buffers
-//   warps 2..5  thread = one token (TMEM lane)
+//   warp 1      MMA issue into a ring of accumulator buffers (three when the head columns fit
+//               three times into 256 tensor-memory columns, else two)
+//   warps 2..9  thread = one token (TMEM lane); warps 2..5 take the even tiles, warps 6..9 the
+//               odd ones.  With three buffers the product of a set's next tile is finished
+//               before the set is done with its current one, so the hand-over (barrier, MMA
+//               issue: several hundred cycles measured) is off the critical path
 // Split-K pieces of a unit leave their candidate in global memory; the piece that arrives last
 // (atomic ticket, nobody waits) picks the winner.  Every barrier wait is bounded.
 #include "sq_decode_common.cuh"
@@ -26,7 +30,8 @@ using namespace tc;
 namespace {
 constexpr int kD = 64;
 constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K tile
-constexpr int kTmemCols = 256;            // two S^T buffers of up to 128 head columns
+constexpr int kTmemCols = 256;            // S^T buffers: 3 x up to 80 or 2 x up to 128 head columns
+constexpr int kGainThreads = 320;         // TMA warp, MMA warp, 2 x 4 token warps
 __host__ __device__ constexpr uint32_t idesc_n(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
@@ -37,20 +42,21 @@ struct Candidate {
 }  // namespace
 
 template <int STAGES>
-__global__ void __launch_bounds__(192, 2)
+__global__ void __launch_bounds__(kGainThreads, 2)
     h2o_gain_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, DecodeArgs a,
-                       int n_cols) {
+                       int n_cols, int n_buf) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = smem;                    // up to 128 head rows
   unsigned char* k_s = q_s + kTM * 128;         // STAGES tiles
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(k_s + STAGES * kTileBytes);
-  static_assert(5 + 2 * STAGES <= 16, "barrier block");
+  static_assert(7 + 2 * STAGES <= 16, "barrier block");
   const uint32_t bar_q = s_u32(bars + 0);
   auto bar_sfull = [&](int j) { return s_u32(bars + 1 + j); };
-  auto bar_sfree = [&](int j) { return s_u32(bars + 3 + j); };
-  auto bar_full = [&](int s) { return s_u32(bars + 5 + s); };
-  auto bar_empty = [&](int s) { return s_u32(bars + 5 + STAGES + s); };
+  auto bar_sfree = [&](int j) { return s_u32(bars + 4 + j); };
+  auto bar_full = [&](int s) { return s_u32(bars + 7 + s); };
+  auto bar_empty = [&](int s) { return s_u32(bars + 7 + STAGES + s); };
+  const int buf_cols = (n_buf == 3) ? n_cols : 128;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* s_nlse = reinterpret_cast<float*>(bars + 18);                     // [128] minus the row log-sum-exp
@@ -77,7 +83,7 @@ __global__ void __launch_bounds__(192, 2)
 
   if (tid == 0) {
     mbar_init(bar_q, 1);
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < 3; ++j) {
       mbar_init(bar_sfull(j), 1);
       mbar_init(bar_sfree(j), 4);  // one arrival per token warp
     }
@@ -93,7 +99,7 @@ __global__ void __launch_bounds__(192, 2)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid >= 64) {
+  if (tid >= 64 && tid < 64 + kTM) {
     const int h = tid - 64;
     // columns past the group read +inf here, so their weight is exp2(-inf) = 0
     s_nlse[h] = (h < G) ? -lse[h] : -INFINITY;
@@ -130,16 +136,16 @@ __global__ void __launch_bounds__(192, 2)
     const uint32_t id = idesc_n(n_cols);
     bool ok = mbar_wait(bar_q, 0, abort_flag);
     for (int i = 0; ok && i < n_tiles; ++i) {
-      const int st = i % STAGES, j = i & 1;
+      const int st = i % STAGES, use = i / n_buf, j = i - use * n_buf;
       ok = mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag);
-      if (ok && i >= 2) ok = mbar_wait(bar_sfree(j), ((i >> 1) - 1) & 1, abort_flag);
+      if (ok && use >= 1) ok = mbar_wait(bar_sfree(j), (use - 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
         const uint32_t k_addr = s_u32(k_s + st * kTileBytes);
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k)
-          umma_bf16(tmem_base + j * 128, umma_desc(k_addr + k * 32), umma_desc(q_addr + k * 32), id, k > 0 ? 1u : 0u);
+          umma_bf16(tmem_base + j * buf_cols, umma_desc(k_addr + k * 32), umma_desc(q_addr + k * 32), id, k > 0 ? 1u : 0u);
         umma_commit(bar_empty(st));
         umma_commit(bar_sfull(j));
       }
@@ -147,7 +153,7 @@ __global__ void __launch_bounds__(192, 2)
     }
   } else {
     // ---------------- thread = one token ----------------
-    const int quarter = warp & 3;
+    const int quarter = warp & 3, set = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
     const int n32 = G >> 5, n8 = ((G & 31) + 7) >> 3;
@@ -155,8 +161,8 @@ __global__ void __launch_bounds__(192, 2)
     unsigned long long best = ~0ull;
     int best_slot = -1;
     bool ok = true;
-    for (int i = 0; ok && i < n_tiles; ++i) {
-      const int j = i & 1;
+    for (int i = set; ok && i < n_tiles; i += 2) {
+      const int use = i / n_buf, j = i - use * n_buf;
       const int slot = t0 + i * kTM + row;
       const bool valid = slot < t1;
       // the score and position loads overlap the wait for the accumulator
@@ -166,23 +172,34 @@ __global__ void __launch_bounds__(192, 2)
         old = acc[slot];
         if (full) p = pos[slot];
       }
-      ok = __all_sync(kFull, mbar_wait(bar_sfull(j), (i >> 1) & 1, abort_flag));  // tcgen05.ld is warp-wide
+      ok = __all_sync(kFull, mbar_wait(bar_sfull(j), use & 1, abort_flag));  // tcgen05.ld is warp-wide
       if (!ok) break;
       tc_fence_after();
-      const uint32_t s_addr = tmem_base + lane_sel + j * 128;
+      const uint32_t s_addr = tmem_base + lane_sel + j * buf_cols;
       float g0 = 0.f, g1 = 0.f;
-#pragma unroll 1
-      for (int ch = 0; ch < n32; ++ch) {
-        float v[32];
-        tmem_ld32(s_addr + ch * 32, v);
+      auto add32 = [&](const uint32_t (&r)[32], int ch) {
         const float4* nl = reinterpret_cast<const float4*>(s_nlse + ch * 32);
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4) {
           const float4 l4 = nl[q4];
-          g0 += ex2(fmaf(v[q4 * 4], c, l4.x));
-          g1 += ex2(fmaf(v[q4 * 4 + 1], c, l4.y));
-          g0 += ex2(fmaf(v[q4 * 4 + 2], c, l4.z));
-          g1 += ex2(fmaf(v[q4 * 4 + 3], c, l4.w));
+          g0 += ex2(fmaf(__uint_as_float(r[q4 * 4]), c, l4.x));
+          g1 += ex2(fmaf(__uint_as_float(r[q4 * 4 + 1]), c, l4.y));
+          g0 += ex2(fmaf(__uint_as_float(r[q4 * 4 + 2]), c, l4.z));
+          g1 += ex2(fmaf(__uint_as_float(r[q4 * 4 + 3]), c, l4.w));
+        }
+      };
+      // the next chunk's tensor-memory load is in flight while this one is summed
+      uint32_t ra[32], rb[32];
+      tmem_ld32_nowait(s_addr, ra);
+#pragma unroll 1
+      for (int ch = 0; ch < n32; ch += 2) {
+        tmem_wait_ld(ra);
+        if (ch + 1 < n32) tmem_ld32_nowait(s_addr + (ch + 1) * 32, rb);
+        add32(ra, ch);
+        if (ch + 1 < n32) {
+          tmem_wait_ld(rb);
+          if (ch + 2 < n32) tmem_ld32_nowait(s_addr + (ch + 2) * 32, ra);
+          add32(rb, ch + 1);
         }
       }
 #pragma unroll 1
@@ -224,8 +241,8 @@ __global__ void __launch_bounds__(192, 2)
       }
     }
     if (lane == 0) {
-      s_cand[quarter].rank = best;
-      s_cand[quarter].slot = best_slot;
+      s_cand[set * 4 + quarter].rank = best;
+      s_cand[set * 4 + quarter].slot = best_slot;
     }
   }
   tc_fence_before();
@@ -241,7 +258,7 @@ __global__ void __launch_bounds__(192, 2)
   }
   if (!full) return;  // the cache still grows: the next token takes a fresh slot
   Candidate best = s_cand[0];
-  for (int q = 1; q < 4; ++q)
+  for (int q = 1; q < 8; ++q)
     if (s_cand[q].rank < best.rank) best = s_cand[q];
   int* victim = reinterpret_cast<int*>(a.pool + ldp->victim_off) + unit;
   if (it.n_split == 1) {
@@ -280,7 +297,7 @@ cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_byt
   if (!make_tile_map(&tm_q, a.q, (long long)q_rows, kD, n_cols) || !make_tile_map(&tm_k, a.pool, pool_rows, kD, kTM))
     return cudaErrorNotSupported;
   constexpr int kStages = 4;
-  constexpr size_t smem = 1024 + (size_t)kTM * 128 + (size_t)kStages * kTileBytes + 18 * 8 + kTM * 4 + 4 * sizeof(Candidate);
+  constexpr size_t smem = 1024 + (size_t)kTM * 128 + (size_t)kStages * kTileBytes + 18 * 8 + kTM * 4 + 8 * sizeof(Candidate);
   auto kern = h2o_gain_tc_kernel<kStages>;
   static bool configured = false;
   if (!configured) {
@@ -288,7 +305,7 @@ cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_byt
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<n_items, 192, smem, s>>>(tm_q, tm_k, a, n_cols);
+  kern<<<n_items, kGainThreads, smem, s>>>(tm_q, tm_k, a, n_cols, 3 * n_cols <= kTmemCols ? 3 : 2);
   return cudaGetLastError();
 }
 
