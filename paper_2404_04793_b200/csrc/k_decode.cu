@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(128, GT == 1 ? 7 : 1) decode_attn_kernel(Decod
       if (h2o) reinterpret_cast<float*>(a.pool + ldp->acc_off)[(size_t)unit * cap + w] = 0.f;
     }
   }
-  if (!h2o && it.n_split > 1) merge_if_last<T>(a, it, unit);
+  if (!h2o && it.n_split > 1) merge_if_last<T, (GT == 1 ? 2 : 4)>(a, it, unit);
 }
 
 // One CTA per (layer, unit): merges the split-K partials into the output and, for H2O, adds

@@ -444,7 +444,6 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     // a shared-memory pipeline (2 per SM) and pay a fixed set-up per CTA, so they want few,
     // long pieces.
     const bool tensor = cfg.dtype == SQ_BF16 && G > 1;
-    const bool wide = tensor && cfg.head_dim == 64 && G > 32;  // 128-token tiles
     const long long target = tensor ? 6LL * c->n_sm : 4LL * c->n_sm;
     if ((long long)U * (e - s) < target / 2)
       split = (int)std::max<long long>(tensor ? 256 : 2 * kMinSplitTokens, (total + target - 1) / target);
