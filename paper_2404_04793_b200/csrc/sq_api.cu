@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -436,23 +437,58 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     int e = s + 1;
     while (e < layer_end && c->n_tok[e] == c->n_tok[s]) ++e;
     const int n_tok = c->n_tok[s];
-    long long total = 0;
-    for (int l = s; l < e; ++l) total += (long long)U * std::min(n_tok + 1, c->hs->layers[l].b);
-    int split = 1 << 30;
-    // Split-K only when the units alone cannot fill the GPU.  How many CTAs that takes depends on
-    // the kernel: the fp32-pipe kernel is light (7 CTAs per SM), the tensor-core kernels carry
-    // a shared-memory pipeline (2 per SM) and pay a fixed set-up per CTA, so they want few,
-    // long pieces.
-    const bool tensor = cfg.dtype == SQ_BF16 && G > 1;
-    const long long target = tensor ? 6LL * c->n_sm : 4LL * c->n_sm;
-    if ((long long)U * (e - s) < target / 2)
-      split = (int)std::max<long long>(tensor ? 256 : 2 * kMinSplitTokens, (total + target - 1) / target);
+    // Split-K plan.  A piece costs a fixed set-up plus its tiles, and pieces run in waves of
+    // as many CTAs as fit the GPU at once; among the piece lengths that are whole tiles, take
+    // the one with the smallest estimated time.  What a tile, a set-up (in tiles; fitted to
+    // measured step times, it includes writing and merging the partial results) and a wave are
+    // depends on the kernel the shape is served by.
+    const bool bf16 = cfg.dtype == SQ_BF16;
+    int tile, setup, per_sm;
+    if (bf16 && cfg.head_dim == 64 && G > 32) {  // tcgen05 kernel: 128-token tiles, 2 CTAs per SM
+      tile = 128, setup = 8, per_sm = 2;
+    } else if (bf16 && G > 1) {                  // mma.sync kernel: 64-token tiles
+      tile = 64, setup = 12, per_sm = cfg.head_dim == 64 && G <= 32 ? 3 : 2;
+    } else {                                     // fp32-pipe kernel
+      tile = 128, setup = 1, per_sm = G == 1 ? 7 : 2;
+    }
+    const long long slots = (long long)per_sm * c->n_sm;
+    int max_len = 1;
+    for (int l = s; l < e; ++l) max_len = std::max(max_len, std::min(n_tok + 1, c->hs->layers[l].b));
+    int split = 0;
+    double best_cost = 0.0;
+    int prev = -1;
+    static const int forced = [] {  // SQ_SPLIT_PIECES=n forces n pieces per longest unit (for measurements)
+      const char* e = getenv("SQ_SPLIT_PIECES");
+      return e ? atoi(e) : 0;
+    }();
+    for (int pieces = 1; pieces <= 64; ++pieces) {
+      int cand = ((max_len + pieces - 1) / pieces + tile - 1) / tile * tile;
+      if (pieces > 1 && cand < 2 * tile) break;  // a piece is never shorter than two tiles
+      if (cand == prev) continue;
+      prev = cand;
+      long long items = 0, work = 0;
+      for (int l = s; l < e; ++l) {
+        const int len = std::min(n_tok + 1, c->hs->layers[l].b);
+        const int ns = (len + cand - 1) / cand;
+        items += (long long)U * ns;
+        work += (long long)U * ((long long)ns * setup + (len + tile - 1) / tile);
+      }
+      if ((size_t)items > c->wl.items_cap) break;
+      // CTAs start in item order, longest layers first: the makespan is about the evenly spread
+      // work, but never below the longest piece, and whole waves when there are only a few
+      const long long waves = (items + slots - 1) / slots;
+      const double t_max = setup + (double)std::min(cand, max_len) / tile;
+      const double spread = (double)work / (double)slots + 0.5 * t_max;
+      const double cost = items <= slots ? t_max : std::max(t_max, std::min(spread, (double)waves * t_max));
+      if (forced > 0 ? (pieces <= forced) : (split == 0 || cost < best_cost * 0.97)) {  // more pieces only for a clear gain
+        best_cost = cost;
+        split = cand;
+      }
+    }
     long long n_items = 0;
-    bool any_split = false;
     for (int l = s; l < e; ++l) {
       int len = std::min(n_tok + 1, c->hs->layers[l].b);
       int ns = (len + split - 1) / split;
-      any_split |= ns > 1;
       n_items += (long long)U * ns;
     }
     if ((size_t)n_items > c->wl.items_cap) return fail(c, SQ_ERR_CAPACITY, "workspace too small for the split plan");

@@ -10,8 +10,7 @@ namespace sq {
 
 constexpr int kMaxLayers = 256;
 constexpr int kMaxGroup = 128;          // query heads per KV head
-constexpr int kMinSplitTokens = 64;     // a split-K piece is never shorter than this (256 for the tcgen05 kernel)
-constexpr int kTargetItems = 148 * 16;  // decode CTAs wanted per launch before split-K stops
+constexpr int kTargetItems = 148 * 16;  // room for split-K pieces beyond one per (layer, unit)
 
 // Per-layer cache geometry, resident in device memory once the budgets are known.
 // k/v/pos/acc/victim offsets are BYTES from the pool base; logit_off counts floats from the
