@@ -72,10 +72,24 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
         step()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        step()
-    e1.record()
+    if per_layer:
+        # one launch per layer is CPU-bound when issued from Python: time a CUDA-graph replay of
+        # the same launches instead (kernel arguments frozen at capture; the caches are full, so
+        # every replay does the same work)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(steps):
+                step()
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+    else:
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     e = 2 if w.dtype == torch.bfloat16 else 4
