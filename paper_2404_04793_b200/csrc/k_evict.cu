@@ -1,25 +1,58 @@
 // C_seq(K, b) on its own (Section 4.1): compresses a layer's cache in place to a tighter
-// budget.  One CTA per unit: decide which slots stay (Sliding Window / StreamingLLM by
-// position, H2O by radix select over the scores), then close the gaps by moving the kept rows
-// towards slot 0 in slot order, 32 slots at a time through shared memory (a row's new slot is
-// never behind its old one, so a tile can be written once it has been read).
+// budget.  One CTA per (unit, layer) of the call:
+//   1. decide which slots stay (Sliding Window / StreamingLLM by position, H2O by radix select
+//      over the scores) and record the decisions as a bitmask in shared memory with a running
+//      count per 32 slots, so that any thread knows a row's new slot without touching memory;
+//   2. close the gaps by moving the kept rows towards slot 0 in slot order.  A row's new slot
+//      is never behind its old one, so reads may run ahead of writes freely: chunks of rows
+//      stream through a multi-stage cp.async ring (rows, positions and scores alike) and are
+//      stored to their new slots when they land.  Only the store of a chunk must follow the
+//      loads of the chunks before it, which the ring order guarantees.
 #include "sq_device.cuh"
 #include "sq_internal.h"
 #include "sq_select.cuh"
 
 namespace sq {
 
-constexpr int kTile = 32;
-constexpr int kMaxVecPerRow = 32;  // 512-byte rows (fp32, head_dim 128)
+namespace {
+constexpr int kChunkBytes = 32 * 1024;  // K and V rows of one chunk
+constexpr int kStages = 3;              // 96 KB of rows in flight per CTA, two CTAs per SM
+constexpr int kMaxVecPerRow = 32;       // 512-byte rows (fp32, head_dim 128)
+constexpr int kMaxChunkRows = kChunkBytes / (2 * 128);  // 128-byte rows (bf16, head_dim 64)
 
+__device__ __forceinline__ void cp_async(void* dst_smem, const void* src, int bytes16) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst_smem);
+  if (bytes16)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src));
+  else
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(src));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
+__device__ __forceinline__ void cp_async_wait_all_but(int n) {
+  switch (n) {
+    case 0: asm volatile("cp.async.wait_group 0;"); break;
+    case 1: asm volatile("cp.async.wait_group 1;"); break;
+    default: asm volatile("cp.async.wait_group 2;"); break;
+  }
+}
+}  // namespace
+
+// Dynamic shared memory: kStages chunks of rows, then per stage the chunk's positions and
+// scores, then the keep bitmask (one word per 32 slots) and its running count.
 __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
+  extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ SelScratch sc;
-  __shared__ uint4 stage[kTile * 2 * kMaxVecPerRow];
-  __shared__ int s_dst[kTile], s_pos[kTile];
-  __shared__ float s_acc[kTile];
+  uint4* stage = reinterpret_cast<uint4*>(dyn);
+  int* s_pos = reinterpret_cast<int*>(dyn + (size_t)kStages * kChunkBytes);
+  float* s_acc = reinterpret_cast<float*>(s_pos + kStages * kMaxChunkRows);
+  unsigned* s_mask = reinterpret_cast<unsigned*>(s_acc + kStages * kMaxChunkRows);
   const int unit = blockIdx.x, tid = threadIdx.x;
-  const LayerDesc& lo = a.ld_old;
-  const int cap = lo.cap, n = a.len, b = a.ld_new.b;
+  const EvictLayer& ev = a.tab[blockIdx.y];
+  const LayerDesc& lo = ev.ld_old;
+  const LayerDesc& ln = ev.ld_new;
+  const int cap = lo.cap, n = ev.len, b = ln.b, n_tok = ev.n_tok;
+  const int n_words = (n + 31) / 32;
+  int* s_before = reinterpret_cast<int*>(s_mask + (cap + 31) / 32);  // kept slots before each word
   int* pos = reinterpret_cast<int*>(a.pool + lo.pos_off) + (size_t)unit * cap;
   float* acc = reinterpret_cast<float*>(a.pool + lo.acc_off) + (size_t)unit * cap;
   const bool h2o = (a.policy == SQ_POLICY_H2O);
@@ -32,18 +65,18 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
   int pos_thr = -1;
   bool heavy = false;
   if (a.policy == SQ_POLICY_SLIDING_WINDOW) {
-    recent_from = a.n_tok - b;
+    recent_from = n_tok - b;
   } else if (a.policy == SQ_POLICY_STREAMING_LLM) {
     n_sink = min(a.n_sink, b);
-    recent_from = a.n_tok - (b - n_sink);
+    recent_from = n_tok - (b - n_sink);
   } else {
-    recent_from = a.n_tok - a.ld_new.b_recent;
-    heavy = a.ld_new.b_heavy > 0;
+    recent_from = n_tok - ln.b_recent;
+    heavy = ln.b_heavy > 0;
     if (heavy) {
       auto key = [&](int i) { return score_key(acc[i]); };
       auto cand = [&](int i) { return pos[i] < recent_from; };
       unsigned int n_at, ties;
-      thr = block_radix_select(sc, n, (unsigned)a.ld_new.b_heavy, key, cand, &n_at, &ties);
+      thr = block_radix_select(sc, n, (unsigned)ln.b_heavy, key, cand, &n_at, &ties);
       if (ties == n_at) {
         pos_thr = 0x7fffffff;
       } else {
@@ -56,64 +89,99 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
     }
   }
 
-  // --- stable compaction ---
-  const int vpr = a.row_bytes / 16;
+  // --- 1. keep bitmask and running counts ---
+  for (int w0 = (tid >> 5); w0 < n_words; w0 += kSelThreads / 32) {
+    const int slot = w0 * 32 + (tid & 31);
+    bool keep = false;
+    if (slot < n) {
+      const int p = pos[slot];
+      if (p >= recent_from || p < n_sink) {
+        keep = true;
+      } else if (heavy) {
+        const uint32_t kk = score_key(acc[slot]);
+        keep = (kk > thr) || (kk == thr && p <= pos_thr);
+      }
+    }
+    const unsigned bal = __ballot_sync(0xffffffffu, keep);
+    if ((tid & 31) == 0) s_mask[w0] = bal;
+  }
+  __syncthreads();
+  if (tid < 32) {  // one warp scans the word counts
+    int running = 0;
+    for (int w0 = 0; w0 < n_words; w0 += 32) {
+      const int w = w0 + tid;
+      const int cnt = (w < n_words) ? __popc(s_mask[w]) : 0;
+      int incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (tid >= o) incl += t;
+      }
+      if (w < n_words) s_before[w] = running + incl - cnt;
+      running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (tid == 0) sc.total = running;
+  }
+  __syncthreads();
+  const int written = sc.total;
+  auto kept = [&](int slot) { return (s_mask[slot >> 5] >> (slot & 31)) & 1u; };
+  auto new_slot = [&](int slot) { return s_before[slot >> 5] + __popc(s_mask[slot >> 5] & ((1u << (slot & 31)) - 1u)); };
+
+  // --- 2. stable compaction through the cp.async ring ---
+  const int vpr = a.row_bytes / 16;                  // 8, 16 or 32 sixteen-byte pieces per row
+  const int lv = 31 - __clz(2 * vpr);                // a slot's K and V pieces: 1 << lv
+  const int rows = kChunkBytes / (2 * a.row_bytes);  // slots per chunk
+  const int n_chunks = (n + rows - 1) / rows;
   uint4* kb = reinterpret_cast<uint4*>(a.pool + lo.k_off) + (size_t)unit * cap * vpr;
   uint4* vb = reinterpret_cast<uint4*>(a.pool + lo.v_off) + (size_t)unit * cap * vpr;
-  int written = 0;
-  for (int s0 = 0; s0 < n; s0 += kTile) {
-    if (tid < 32) {
-      const int slot = s0 + tid;
-      bool keep = false;
-      int p = -1;
-      float sc_v = 0.f;
-      if (slot < n) {
-        p = pos[slot];
-        if (h2o) sc_v = acc[slot];
-        if (p >= recent_from || p < n_sink) {
-          keep = true;
-        } else if (heavy) {
-          uint32_t kk = score_key(sc_v);
-          keep = (kk > thr) || (kk == thr && p <= pos_thr);
+  auto issue = [&](int c) {
+    if (c < n_chunks) {
+      const int s0 = c * rows, st = c % kStages;
+      uint4* sg = stage + (size_t)st * (kChunkBytes / 16);
+      for (int idx = tid; idx < rows * 2 * vpr; idx += kSelThreads) {
+        const int j = idx >> lv, r = idx & ((1 << lv) - 1);
+        const int slot = s0 + j;
+        if (slot >= n || !kept(slot)) continue;
+        const size_t src = (size_t)slot * vpr;
+        cp_async(sg + idx, (r < vpr) ? (kb + src + r) : (vb + src + r - vpr), 1);
+        if (r == 0) {
+          cp_async(s_pos + st * kMaxChunkRows + j, pos + slot, 0);
+          if (h2o) cp_async(s_acc + st * kMaxChunkRows + j, acc + slot, 0);
         }
       }
-      const unsigned bal = __ballot_sync(0xffffffffu, keep);
-      s_dst[tid] = keep ? written + __popc(bal & ((1u << tid) - 1u)) : -1;
-      s_pos[tid] = p;
-      s_acc[tid] = sc_v;
-      if (tid == 0) sc.total = __popc(bal);
     }
+    cp_async_commit();  // one group per chunk, empty past the end, so the wait counts stay aligned
+  };
+  for (int c = 0; c < kStages - 1; ++c) issue(c);
+  for (int c = 0; c < n_chunks; ++c) {
+    issue(c + kStages - 1);
+    cp_async_wait_all_but(kStages - 1);
     __syncthreads();
-    for (int idx = tid; idx < kTile * 2 * vpr; idx += kSelThreads) {
-      const int j = idx / (2 * vpr), r = idx - j * 2 * vpr;
-      if (s_dst[j] < 0) continue;
-      const size_t src = (size_t)(s0 + j) * vpr;
-      stage[idx] = (r < vpr) ? kb[src + r] : vb[src + r - vpr];
-    }
-    __syncthreads();
-    for (int idx = tid; idx < kTile * 2 * vpr; idx += kSelThreads) {
-      const int j = idx / (2 * vpr), r = idx - j * 2 * vpr;
-      const int d = s_dst[j];
-      if (d < 0) continue;
+    const int s0 = c * rows, st = c % kStages;
+    const uint4* sg = stage + (size_t)st * (kChunkBytes / 16);
+    for (int idx = tid; idx < rows * 2 * vpr; idx += kSelThreads) {
+      const int j = idx >> lv, r = idx & ((1 << lv) - 1);
+      const int slot = s0 + j;
+      if (slot >= n || !kept(slot)) continue;
+      const int d = new_slot(slot);
       if (d >= b) {
         atomicOr(a.status, 4);
         continue;
       }
-      if (r < vpr) kb[(size_t)d * vpr + r] = stage[idx];
-      else vb[(size_t)d * vpr + r - vpr] = stage[idx];
+      if (r < vpr) kb[(size_t)d * vpr + r] = sg[idx];
+      else vb[(size_t)d * vpr + r - vpr] = sg[idx];
       if (r == 0) {
-        pos[d] = s_pos[j];
-        if (h2o) acc[d] = s_acc[j];
+        pos[d] = s_pos[st * kMaxChunkRows + j];
+        if (h2o) acc[d] = s_acc[st * kMaxChunkRows + j];
       }
     }
-    written += sc.total;
-    __syncthreads();
+    __syncthreads();  // the stage is refilled by the next iteration's loads
   }
   if (tid == 0 && written != b) atomicOr(a.status, 8);
 
   // --- H2O: the slot the next append replaces ---
   if (h2o) {
-    const int vthr = a.n_tok - a.ld_new.b_recent;
+    const int vthr = n_tok - ln.b_recent;
     unsigned long long best = ~0ull;
     int slot = -1;
     for (int i = tid; i < b; i += kSelThreads) {
@@ -132,8 +200,18 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
 }
 
 cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s) {
-  if (a.row_bytes / 16 > kMaxVecPerRow) return cudaErrorInvalidValue;
-  evict_kernel<<<a.n_unit, kSelThreads, 0, s>>>(a);
+  if (a.row_bytes / 16 > kMaxVecPerRow || a.row_bytes < 128 || (a.row_bytes & (a.row_bytes - 1)))
+    return cudaErrorInvalidValue;
+  const size_t words = ((size_t)a.max_cap + 31) / 32;
+  const size_t smem = (size_t)kStages * kChunkBytes + (size_t)kStages * kMaxChunkRows * 8 + words * 8;
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;  // caches beyond ~1.4 M slots per unit
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  evict_kernel<<<dim3(a.n_unit, a.n_layers), kSelThreads, smem, s>>>(a);
   return cudaGetLastError();
 }
 

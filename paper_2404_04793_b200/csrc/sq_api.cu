@@ -21,7 +21,7 @@ inline int elem_bytes(int dtype) { return dtype == SQ_F32 ? 4 : 2; }
 constexpr int kMaxImportanceCtas = 4096;
 
 struct WsLayout {
-  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order;
+  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order, evict_tab;
   size_t part_stat, part_o, logits, acc_prompt, lse2, total;
   size_t items_cap, logits_floats;
 };
@@ -33,6 +33,7 @@ struct HostStage {  // pinned
   long long tok_count[kMaxLayers];
   LayerDesc layers[kMaxLayers];
   int order[kMaxLayers];
+  EvictLayer evict_tab[kMaxLayers];
   int32_t status;
 };
 
@@ -117,6 +118,7 @@ WsLayout ws_layout(const sq_config& c, int64_t b_init) {
   w.tickets = take(4 * L * U);
   w.layers = take(sizeof(LayerDesc) * L);
   w.order = take(4 * L);
+  w.evict_tab = take(sizeof(EvictLayer) * L);
   w.items_cap = (size_t)kTargetItems + U * L;
   w.part_stat = take(w.items_cap * G * 4 * 4);
   w.part_o = take(w.items_cap * G * c.head_dim * 4);
@@ -193,13 +195,6 @@ int ensure_budgets(sq_ctx* c, cudaStream_t st) {
   if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "budgets not set: call sq_allocate_budgets or sq_set_budgets first");
   SQ_CUDA(c, cudaEventSynchronize(c->ev));
   return build_layout(c, st);
-}
-
-int upload_layer(sq_ctx* c, int l, cudaStream_t st) {
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers) + l, &c->hs->layers[l], sizeof(LayerDesc),
-                             cudaMemcpyHostToDevice, st));
-  SQ_CUDA(c, cudaStreamSynchronize(st));
-  return SQ_OK;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -544,6 +539,7 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
       return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
   }
   const int U = c->batch * cfg.n_kv_head;
+  int n_active = 0, max_cap = 0;
   for (int l = layer_begin; l < layer_end; ++l) {
     const int nb = new_budgets_host[l - layer_begin];
     LayerDesc old = c->hs->layers[l];
@@ -567,24 +563,34 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
       }
     }
     if (len > nb) {
-      EvictArgs a;
-      a.pool = c->pool;
-      a.ld_old = old;
-      a.ld_new = nw;
-      a.n_unit = U;
-      a.len = len;
-      a.n_tok = n_tok;
-      a.policy = cfg.policy;
-      a.n_sink = cfg.n_sink;
-      a.row_bytes = cfg.head_dim * elem_bytes(cfg.dtype);
-      a.status = ws_ptr<int>(c, c->wl.status);
-      SQ_CUDA(c, launch_evict(a, st));
+      EvictLayer& e = c->hs->evict_tab[n_active++];
+      e.ld_old = old;
+      e.ld_new = nw;
+      e.len = len;
+      e.n_tok = n_tok;
+      max_cap = std::max(max_cap, old.cap);
     }
     c->hs->layers[l] = nw;
     c->hs->budget[l] = nb;
-    rc = upload_layer(c, l, st);
-    if (rc != SQ_OK) return rc;
   }
+  if (n_active > 0) {
+    // all layers of the call in one launch
+    EvictArgs a;
+    a.pool = c->pool;
+    a.tab = ws_ptr<EvictLayer>(c, c->wl.evict_tab);
+    a.n_layers = n_active;
+    a.max_cap = max_cap;
+    a.n_unit = U;
+    a.policy = cfg.policy;
+    a.n_sink = cfg.n_sink;
+    a.row_bytes = cfg.head_dim * elem_bytes(cfg.dtype);
+    a.status = ws_ptr<int>(c, c->wl.status);
+    SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<EvictLayer>(c, c->wl.evict_tab), c->hs->evict_tab, sizeof(EvictLayer) * n_active,
+                               cudaMemcpyHostToDevice, st));
+    SQ_CUDA(c, launch_evict(a, st));
+  }
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers) + layer_begin, &c->hs->layers[layer_begin],
+                             sizeof(LayerDesc) * (layer_end - layer_begin), cudaMemcpyHostToDevice, st));
   // the launch order (largest budget first) may have changed
   std::vector<int> ord(cfg.n_layer);
   for (int l = 0; l < cfg.n_layer; ++l) ord[l] = l;

@@ -89,10 +89,16 @@ struct DecodeArgs {
   float scale_log2;  // log2(e) / sqrt(head_dim)
 };
 
+struct EvictLayer {  // one layer of an explicit eviction
+  LayerDesc ld_old, ld_new;
+  int len, n_tok;
+};
+
 struct EvictArgs {
   char* pool;
-  LayerDesc ld_old, ld_new;
-  int n_unit, len, n_tok, policy, n_sink, row_bytes;
+  const EvictLayer* tab;  // [n_layers] in device memory
+  int n_layers, max_cap;
+  int n_unit, policy, n_sink, row_bytes;
   int* status;
 };
 

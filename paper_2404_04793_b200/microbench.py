@@ -124,6 +124,33 @@ def prefill_compress_time(w: synth.Workload, reps=3, device="cuda:0"):
                 causal_score_flops=flops, tflops=round(flops / ms / 1e9, 1), device_status=ctx.status())
 
 
+def touch_all_kernels(w: synth.Workload, device="cuda:0"):
+    """One short pass that launches every kernel of the library on a workload (importance,
+    allocator, prefill scoring / selection / gather, decode steps, explicit eviction to half the
+    budgets): the command behind the per-kernel profiler summaries."""
+    job = engine.Job(w, device)
+    ctx = job.ctx
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    for l in range(w.n_layer):
+        a, b = synth.hidden_pair(w, l, device)
+        ctx.layer_importance(l, a, b)
+        del a, b
+    ctx.allocate_budgets(w.b_init, w.p)
+    budgets, _ = ctx.get_budgets()
+    for l in range(w.n_layer):
+        q, k, v = synth.prompt_qkv(w, l, device, need_q=(w.policy == synth.H2O))
+        ctx.prefill_compress(l, k, v, q)
+        del q, k, v
+    for t in range(w.steps):
+        q, kn, vn = synth.decode_qkv(w, t, device)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+    floor = (w.n_sink + 1) if w.policy == synth.STREAMING_LLM else 1
+    ctx.evict(0, w.n_layer, [max(floor, b // 2) for b in budgets])
+    torch.cuda.synchronize()
+    return dict(workload=w.name, what="every kernel once", budgets=budgets, device_status=ctx.status())
+
+
 def generation_throughput(w: synth.Workload, device="cuda:0"):
     """Decode tokens/s of the attention + eviction path over a whole generation: cache filled
     from a prompt of w.prompt tokens, then w.steps fused decode steps, all timed together."""
@@ -197,11 +224,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
+    ap.add_argument("--all-kernels", action="store_true", help="launch every kernel of the library once or a few times")
+    ap.add_argument("--layers", type=int, default=0, help="with --all-kernels: number of layers of the shape to keep")
     ap.add_argument("--compare-budgets", action="store_true",
                     help="generation throughput: full cache vs sequence-wise policy alone vs layer-wise budgets")
     ap.add_argument("--sweep-falcon", action="store_true",
                     help="decode-step time over the Falcon-7B-shaped grid: batch x prompt x budget x policy")
     args = ap.parse_args()
+    if args.all_kernels:
+        w = build_workload(args)
+        kw = dict(steps=args.steps)
+        if args.layers:
+            kw["n_layer"] = args.layers
+        print(json.dumps(touch_all_kernels(w.replace(**kw))), flush=True)
+        return
     if args.compare_budgets:
         compare_budgets()
         return
