@@ -80,6 +80,16 @@ typedef struct sq_config {
   int32_t heavy_den;      /*      budget b go to heavy hitters, the rest to recent tokens   */
   int32_t n_cluster;      /* 3 (Algorithm 1, step 5) or 2                                   */
   int32_t page_tokens;    /* per-unit slot ranges are rounded up to this many tokens (>= 1) */
+  int32_t per_sequence_budgets; /* 0: one budget vector for the batch, from the cosine averaged over
+                                      all its prompts (the default);  1: one budget vector per
+                                      prompt (Section 4.1 allocates "for the given prompt"): every
+                                      sequence is clustered on its own averages and gets its own
+                                      per-layer budgets, each summing to n_layer * b_init.  Then the
+                                      per-layer arrays of sq_set_budgets, sq_get_cos_sim,
+                                      sq_get_budgets and sq_evict are [batch][n_layer] (sequence
+                                      first), sq_layer_importance takes the rows sequence by
+                                      sequence (prompt_len rows each, all of them before
+                                      sq_allocate_budgets), and decode launches are not split-K */
 } sq_config;
 
 /* Bytes of cache pool and workspace a context needs when the per-layer budgets sum to at most

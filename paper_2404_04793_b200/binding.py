@@ -32,7 +32,8 @@ EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequen
 class sq_config(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in (
         "n_layer", "n_q_head", "n_kv_head", "head_dim", "hidden", "max_batch", "max_prompt",
-        "max_new_tokens", "dtype", "policy", "n_sink", "heavy_num", "heavy_den", "n_cluster", "page_tokens")]
+        "max_new_tokens", "dtype", "policy", "n_sink", "heavy_num", "heavy_den", "n_cluster", "page_tokens",
+        "per_sequence_budgets")]
 
 
 class SqError(RuntimeError):
@@ -96,10 +97,11 @@ def _stream():
 
 
 def make_config(*, n_layer, n_q_head, n_kv_head, head_dim, hidden, max_batch, max_prompt, max_new_tokens,
-                dtype, policy, n_sink=4, heavy_num=1, heavy_den=2, n_cluster=3, page_tokens=16) -> sq_config:
+                dtype, policy, n_sink=4, heavy_num=1, heavy_den=2, n_cluster=3, page_tokens=16,
+                per_sequence_budgets=0) -> sq_config:
     dt = {torch.float32: SQ_F32, torch.bfloat16: SQ_BF16}.get(dtype, dtype)
     return sq_config(n_layer, n_q_head, n_kv_head, head_dim, hidden, max_batch, max_prompt, max_new_tokens,
-                     dt, policy, n_sink, heavy_num, heavy_den, n_cluster, page_tokens)
+                     dt, policy, n_sink, heavy_num, heavy_den, n_cluster, page_tokens, int(per_sequence_budgets))
 
 
 def sq_query_sizes(cfg: sq_config, b_init: int):
@@ -112,7 +114,8 @@ def sq_query_sizes(cfg: sq_config, b_init: int):
 
 class Context:
     """One libsq context plus the device memory it lives in (two torch byte tensors).
-    Methods carry the C names without the sq_ prefix and take torch CUDA tensors."""
+    Methods carry the C names without the sq_ prefix and take torch CUDA tensors.  With
+    per_sequence_budgets the per-layer lists become lists of per-sequence lists ([batch][n_layer])."""
 
     def __init__(self, cfg: sq_config, b_init: int, device="cuda:0"):
         self.cfg = cfg
@@ -148,6 +151,7 @@ class Context:
             raise SqError(rc, lib().sq_last_error(self._h).decode())
 
     def begin_sequence_batch(self, batch, prompt_len):
+        self.batch = int(batch)
         self._ck(lib().sq_begin_sequence_batch(self._h, batch, prompt_len, _stream()))
 
     def layer_importance(self, layer, hidden_in, hidden_out):
@@ -157,8 +161,28 @@ class Context:
     def allocate_budgets(self, b_init, p):
         self._ck(lib().sq_allocate_budgets(self._h, int(b_init), float(p), _stream()))
 
+    def _rows(self):
+        return self.batch if self.cfg.per_sequence_budgets else 1
+
+    def _flatten(self, values, n):
+        """[n] -> [n]; with per-sequence budgets [batch][n] -> the C layout (sequence first)."""
+        if self.cfg.per_sequence_budgets:
+            if len(values) != self.batch or any(len(v) != n for v in values):
+                raise ValueError("expected one list per sequence")
+            return [int(b) for row in values for b in row]
+        if len(values) != n:
+            raise ValueError("expected one value per layer")
+        return [int(b) for b in values]
+
+    def _nest(self, flat, n):
+        flat = list(flat)
+        if self.cfg.per_sequence_budgets:
+            return [flat[s * n:(s + 1) * n] for s in range(self.batch)]
+        return flat
+
     def set_budgets(self, budgets):
-        arr = (c_int32 * self.cfg.n_layer)(*[int(b) for b in budgets])
+        flat = self._flatten(budgets, self.cfg.n_layer)
+        arr = (c_int32 * len(flat))(*flat)
         self._ck(lib().sq_set_budgets(self._h, arr, _stream()))
 
     def prefill_compress(self, layer, k_prompt, v_prompt, q_prompt=None, acc_prompt=None):
@@ -170,19 +194,21 @@ class Context:
                                       _dptr(out), _stream()))
 
     def evict(self, layer_begin, layer_end, new_budgets):
-        arr = (c_int32 * (layer_end - layer_begin))(*[int(b) for b in new_budgets])
+        flat = self._flatten(new_budgets, layer_end - layer_begin)
+        arr = (c_int32 * len(flat))(*flat)
         self._ck(lib().sq_evict(self._h, layer_begin, layer_end, arr, _stream()))
 
     def get_cos_sim(self):
-        arr = (c_float * self.cfg.n_layer)()
+        arr = (c_float * (self.cfg.n_layer * self._rows()))()
         self._ck(lib().sq_get_cos_sim(self._h, arr))
-        return torch.tensor(list(arr), dtype=torch.float32)
+        return torch.tensor(self._nest(arr, self.cfg.n_layer), dtype=torch.float32)
 
     def get_budgets(self):
-        b = (c_int32 * self.cfg.n_layer)()
-        g = (c_uint8 * self.cfg.n_layer)()
+        n = self.cfg.n_layer * self._rows()
+        b = (c_int32 * n)()
+        g = (c_uint8 * n)()
         self._ck(lib().sq_get_budgets(self._h, b, g))
-        return list(b), [bool(x) for x in g]
+        return self._nest(b, self.cfg.n_layer), self._nest([bool(x) for x in g], self.cfg.n_layer)
 
     def get_len(self, layer):
         n = c_int32()
@@ -198,12 +224,13 @@ class Context:
         return list(pos[: n.value]), list(acc[: n.value])
 
     def get_kv(self, layer, seq, kv_head):
-        n = self.get_len(layer)
+        cap = self.get_len(layer)                       # the layer's longest unit
+        n = len(self.get_kept(layer, seq, kv_head)[0])  # this unit
         dt = torch.float32 if self.cfg.dtype == SQ_F32 else torch.bfloat16
-        k = torch.empty(n, self.cfg.head_dim, dtype=dt)
-        v = torch.empty(n, self.cfg.head_dim, dtype=dt)
+        k = torch.empty(max(cap, 1), self.cfg.head_dim, dtype=dt)
+        v = torch.empty(max(cap, 1), self.cfg.head_dim, dtype=dt)
         self._ck(lib().sq_get_kv(self._h, layer, seq, kv_head, c_void_p(k.data_ptr()), c_void_p(v.data_ptr())))
-        return k, v
+        return k[:n], v[:n]
 
     def status(self):
         s = c_int32()

@@ -224,12 +224,16 @@ template <typename T>
 __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
   __shared__ SelScratch sc;
   __shared__ __align__(16) float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
-  const int n_layers = a.layer_end - a.layer_begin;
-  const int layer = a.layer_begin + blockIdx.x / a.n_unit;
-  const int unit = blockIdx.x % a.n_unit;
-  (void)n_layers;
+  int layer = a.layer_begin + blockIdx.x / a.n_unit;
+  int unit = blockIdx.x % a.n_unit;
   ItemLoc it;
-  if (!locate(a, 0, layer, it)) return;
+  if (a.uniform) {  // items are (descriptor, unit) pairs in launch order
+    if (!locate(a, blockIdx.x, -1, it)) return;
+    layer = it.layer;
+    unit = it.local;
+  } else if (!locate(a, 0, layer, it)) {
+    return;
+  }
   const int tid = threadIdx.x, D = a.head_dim, G = a.group, ns = it.n_split;
   const LayerDesc* ldp = a.layers + layer;
   const int b = ldp->b, cap = ldp->cap;

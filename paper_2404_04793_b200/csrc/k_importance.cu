@@ -115,12 +115,13 @@ __global__ void __launch_bounds__(256) allocate_budgets_kernel(AllocateArgs a) {
   __shared__ int s_best_id[256];
   __shared__ int s_k, s_cut;
   const int n = a.n_layer, tid = threadIdx.x;
+  const int st = a.stride, off = blockIdx.x;  // this CTA's budget vector: entries i * st + off
 
   // layer averages, rounded to fp32 (the value reported to the caller), ranked by (value, layer)
   for (int i = tid; i < n; i += blockDim.x) {
-    long long cnt = a.tok_count[i];
-    float c = cnt > 0 ? (float)(a.cos_sum[i] / (double)cnt) : 0.f;
-    a.cos_sim[i] = c;
+    long long cnt = a.tok_count[i * st + off];
+    float c = cnt > 0 ? (float)(a.cos_sum[i * st + off] / (double)cnt) : 0.f;
+    a.cos_sim[i * st + off] = c;
     s_head[i] = (double)c;  // scratch: unsorted values
   }
   __syncthreads();
@@ -191,11 +192,11 @@ __global__ void __launch_bounds__(256) allocate_budgets_kernel(AllocateArgs a) {
     const int cut = s_cut;
     const int n3 = n - cut;
     for (int i = 0; i < n; ++i) {
-      a.is_g3[i] = 0;
-      a.budget[i] = (int)a.b_init;
+      a.is_g3[i * st + off] = 0;
+      a.budget[i * st + off] = (int)a.b_init;
     }
     if (n3 > 0 && n3 < n) {
-      for (int r = cut; r < n; ++r) a.is_g3[s_idx[r]] = 1;
+      for (int r = cut; r < n; ++r) a.is_g3[s_idx[r] * st + off] = 1;
       long long b_low = (long long)floor(__dmul_rn((double)a.b_init, a.p));
       if (b_low < 1) b_low = 1;
       long long rest = (long long)n * a.b_init - (long long)n3 * b_low;
@@ -203,10 +204,10 @@ __global__ void __launch_bounds__(256) allocate_budgets_kernel(AllocateArgs a) {
       long long base = rest / m, extra = rest % m;
       long long seen = 0;
       for (int i = 0; i < n; ++i) {
-        if (a.is_g3[i]) {
-          a.budget[i] = (int)b_low;
+        if (a.is_g3[i * st + off]) {
+          a.budget[i * st + off] = (int)b_low;
         } else {
-          a.budget[i] = (int)(base + (seen < extra ? 1 : 0));
+          a.budget[i * st + off] = (int)(base + (seen < extra ? 1 : 0));
           ++seen;
         }
       }
@@ -215,7 +216,7 @@ __global__ void __launch_bounds__(256) allocate_budgets_kernel(AllocateArgs a) {
 }
 
 cudaError_t launch_allocate(const AllocateArgs& a, cudaStream_t s) {
-  allocate_budgets_kernel<<<1, 256, 0, s>>>(a);
+  allocate_budgets_kernel<<<a.stride, 256, 0, s>>>(a);
   return cudaGetLastError();
 }
 

@@ -21,20 +21,25 @@ inline int elem_bytes(int dtype) { return dtype == SQ_F32 ? 4 : 2; }
 constexpr int kMaxImportanceCtas = 4096;
 
 struct WsLayout {
-  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order, evict_tab;
+  size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order, order_by_layer,
+      evict_tab;
   size_t part_stat, part_o, logits, acc_prompt, lse2, total;
-  size_t items_cap, logits_floats;
+  size_t items_cap, logits_floats, n_desc_cap;
 };
 
-struct HostStage {  // pinned
-  int32_t budget[kMaxLayers];
-  uint8_t is_g3[kMaxLayers];
-  float cos_sim[kMaxLayers];
-  long long tok_count[kMaxLayers];
-  LayerDesc layers[kMaxLayers];
-  int order[kMaxLayers];
-  EvictLayer evict_tab[kMaxLayers];
-  int32_t status;
+// Pinned staging for the small host <-> device tables.  "desc" = one cache descriptor: a layer
+// of the whole batch, or with per-sequence budgets a (layer, sequence) pair; arrays hold
+// n_desc_cap entries, entry of (layer, group) = layer * n_grp + group.
+struct HostStage {
+  int32_t* budget;
+  uint8_t* is_g3;
+  float* cos_sim;
+  long long* tok_count;
+  LayerDesc* layers;
+  int* order;           // all descriptors, largest budget first
+  int* order_by_layer;  // per layer its descriptors, largest budget first
+  EvictLayer* evict_tab;
+  void* block;
 };
 
 }  // namespace
@@ -47,13 +52,18 @@ struct sq_ctx {
   char* ws;
   size_t ws_bytes;
   WsLayout wl;
-  HostStage* hs;
+  HostStage hs;
   cudaEvent_t ev;
   int n_sm;
   int batch, prompt;
+  bool per_seq;    // one budget vector per sequence instead of one per batch
+  int n_grp;       // descriptors per layer: batch with per-sequence budgets, else 1
+  int desc_units;  // units (sequence, KV head) per descriptor
+  int n_desc;      // n_layer * n_grp
   bool begun;
   int budget_state;  // 0 none, 1 computed on device (copy in flight), 2 on host, laid out
   int n_tok[kMaxLayers];
+  long long imp_tokens[kMaxLayers];  // tokens of a layer seen by sq_layer_importance so far
   bool prefilled[kMaxLayers];
   bool importance_seen[kMaxLayers];
   std::string err;
@@ -88,6 +98,7 @@ int check_config(const sq_config* c, std::string* why) {
     return bad("H2O needs 0 <= heavy_num < heavy_den");
   if (c->n_cluster != 2 && c->n_cluster != 3) return bad("n_cluster must be 2 or 3");
   if (c->page_tokens < 1) return bad("page_tokens must be >= 1");
+  if (c->per_sequence_budgets != 0 && c->per_sequence_budgets != 1) return bad("per_sequence_budgets must be 0 or 1");
   return SQ_OK;
 }
 
@@ -95,30 +106,34 @@ size_t pool_bytes_for(const sq_config& c, int64_t b_init) {
   const size_t U = (size_t)c.max_batch * c.n_kv_head;
   const size_t tokens = (size_t)c.n_layer * (size_t)b_init + (size_t)c.n_layer * (c.page_tokens - 1);
   size_t per_tok = 2 * (size_t)c.head_dim * elem_bytes(c.dtype) + 4 + (c.policy == SQ_POLICY_H2O ? 4 : 0);
-  return U * tokens * per_tok + (size_t)c.n_layer * (U * 4 + 6 * kAlign);
+  const size_t n_desc = (size_t)c.n_layer * (c.per_sequence_budgets ? c.max_batch : 1);
+  return U * tokens * per_tok + (size_t)c.n_layer * U * 4 + n_desc * 6 * kAlign;
 }
 
 WsLayout ws_layout(const sq_config& c, int64_t b_init) {
   WsLayout w{};
   const size_t L = c.n_layer, U = (size_t)c.max_batch * c.n_kv_head, G = c.n_q_head / c.n_kv_head;
+  const size_t ND = L * (c.per_sequence_budgets ? (size_t)c.max_batch : 1);
+  w.n_desc_cap = ND;
   size_t off = 0;
   auto take = [&](size_t bytes) {
     size_t o = off;
     off = align_up(off + bytes);
     return o;
   };
-  w.cos_sum = take(8 * L);
-  w.tok_count = take(8 * L);
+  w.cos_sum = take(8 * ND);
+  w.tok_count = take(8 * ND);
   w.cta_partial = take(4 * (size_t)kMaxImportanceCtas);
   w.ticket = take(4);
-  w.cos_sim = take(4 * L);
-  w.budget = take(4 * L);
-  w.is_g3 = take(L);
+  w.cos_sim = take(4 * ND);
+  w.budget = take(4 * ND);
+  w.is_g3 = take(ND);
   w.status = take(4);
   w.tickets = take(4 * L * U);
-  w.layers = take(sizeof(LayerDesc) * L);
-  w.order = take(4 * L);
-  w.evict_tab = take(sizeof(EvictLayer) * L);
+  w.layers = take(sizeof(LayerDesc) * ND);
+  w.order = take(4 * ND);
+  w.order_by_layer = take(4 * ND);
+  w.evict_tab = take(sizeof(EvictLayer) * ND);
   w.items_cap = (size_t)kTargetItems + U * L;
   w.part_stat = take(w.items_cap * G * 4 * 4);
   w.part_o = take(w.items_cap * G * c.head_dim * 4);
@@ -143,47 +158,60 @@ T* ws_ptr(sq_ctx* c, size_t off) {
       return fail((c), SQ_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__));        \
   } while (0)
 
-// Computes the per-layer cache geometry for the budgets in hs->budget and uploads it.
+// Launch orders: all descriptors by budget (the fused launch starts the longest first), and
+// the same within each layer (launches over a sub-range of layers).
+void sort_orders(sq_ctx* c) {
+  const int nd = c->n_desc, ng = c->n_grp;
+  std::vector<int> ord(nd);
+  for (int d = 0; d < nd; ++d) ord[d] = d;
+  auto by_budget = [&](int x, int y) { return c->hs.budget[x] > c->hs.budget[y]; };
+  std::stable_sort(ord.begin(), ord.end(), by_budget);
+  std::copy(ord.begin(), ord.end(), c->hs.order);
+  for (int d = 0; d < nd; ++d) ord[d] = d;
+  for (int l = 0; l < c->cfg.n_layer; ++l) std::stable_sort(ord.begin() + l * ng, ord.begin() + (l + 1) * ng, by_budget);
+  std::copy(ord.begin(), ord.end(), c->hs.order_by_layer);
+}
+
+// Computes the cache geometry for the budgets in hs.budget and uploads it.
 int build_layout(sq_ctx* c, cudaStream_t st) {
   const sq_config& cfg = c->cfg;
-  const size_t U = (size_t)c->batch * cfg.n_kv_head, G = cfg.n_q_head / cfg.n_kv_head;
+  const size_t U = (size_t)c->desc_units, G = cfg.n_q_head / cfg.n_kv_head;
   const size_t row = (size_t)cfg.head_dim * elem_bytes(cfg.dtype);
   const bool h2o = cfg.policy == SQ_POLICY_H2O;
   size_t off = 0, lfl = 0;
-  for (int l = 0; l < cfg.n_layer; ++l) {
-    LayerDesc& d = c->hs->layers[l];
-    const int b = c->hs->budget[l];
+  for (int d = 0; d < c->n_desc; ++d) {
+    LayerDesc& ld = c->hs.layers[d];
+    const int b = c->hs.budget[d];
     if (b < 1) return fail(c, SQ_ERR_INVALID_ARG, "a layer budget is below 1");
     if (cfg.policy == SQ_POLICY_STREAMING_LLM && b <= cfg.n_sink)
       return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
-    d.b = b;
-    d.cap = (b + cfg.page_tokens - 1) / cfg.page_tokens * cfg.page_tokens;
-    d.b_heavy = h2o ? (int)(((long long)b * cfg.heavy_num) / cfg.heavy_den) : 0;
-    d.b_recent = b - d.b_heavy;
-    d.ring_base = (cfg.policy == SQ_POLICY_STREAMING_LLM) ? cfg.n_sink : 0;
-    d.ring_origin = std::max(d.ring_base, c->prompt - (b - d.ring_base));
-    d.k_off = (long long)off;
-    off = align_up(off + U * d.cap * row);
-    d.v_off = (long long)off;
-    off = align_up(off + U * d.cap * row);
-    d.pos_off = (long long)off;
-    off = align_up(off + U * d.cap * 4);
-    d.acc_off = (long long)off;
-    if (h2o) off = align_up(off + U * d.cap * 4);
-    d.victim_off = (long long)off;
+    ld.b = b;
+    ld.cap = (b + cfg.page_tokens - 1) / cfg.page_tokens * cfg.page_tokens;
+    ld.b_heavy = h2o ? (int)(((long long)b * cfg.heavy_num) / cfg.heavy_den) : 0;
+    ld.b_recent = b - ld.b_heavy;
+    ld.ring_base = (cfg.policy == SQ_POLICY_STREAMING_LLM) ? cfg.n_sink : 0;
+    ld.ring_origin = std::max(ld.ring_base, c->prompt - (b - ld.ring_base));
+    ld.k_off = (long long)off;
+    off = align_up(off + U * ld.cap * row);
+    ld.v_off = (long long)off;
+    off = align_up(off + U * ld.cap * row);
+    ld.pos_off = (long long)off;
+    off = align_up(off + U * ld.cap * 4);
+    ld.acc_off = (long long)off;
+    if (h2o) off = align_up(off + U * ld.cap * 4);
+    ld.victim_off = (long long)off;
     off = align_up(off + U * 4);
-    d.logit_off = (long long)lfl;
-    if (h2o) lfl += U * d.cap * G;
+    ld.logit_off = (long long)lfl;
+    if (h2o) lfl += U * ld.cap * G;
   }
   if (off > c->pool_bytes) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the cache pool");
   if (lfl > c->wl.logits_floats) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the workspace");
-  std::vector<int> ord(cfg.n_layer);
-  for (int l = 0; l < cfg.n_layer; ++l) ord[l] = l;
-  std::stable_sort(ord.begin(), ord.end(), [&](int x, int y) { return c->hs->budget[x] > c->hs->budget[y]; });
-  std::copy(ord.begin(), ord.end(), c->hs->order);
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers), c->hs->layers, sizeof(LayerDesc) * cfg.n_layer,
+  sort_orders(c);
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers), c->hs.layers, sizeof(LayerDesc) * c->n_desc,
                              cudaMemcpyHostToDevice, st));
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs->order, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs.order, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order_by_layer), c->hs.order_by_layer, 4 * c->n_desc,
+                             cudaMemcpyHostToDevice, st));
   // the staging block is reused by later calls: make sure the copies have left it
   SQ_CUDA(c, cudaStreamSynchronize(st));
   c->budget_state = 2;
@@ -198,6 +226,10 @@ int ensure_budgets(sq_ctx* c, cudaStream_t st) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// User-facing arrays are [n_layer] (one budget vector per batch) or [batch][n_layer]
+// (per-sequence budgets); internally entry (layer, group) sits at layer * n_grp + group.
+inline int user_index(const sq_ctx* c, int layer, int grp) { return grp * c->cfg.n_layer + layer; }
 
 }  // namespace
 
@@ -237,16 +269,37 @@ int sq_ctx_create(const sq_config* cfg, int64_t b_init, void* pool, size_t pool_
   c->ws_bytes = workspace_bytes;
   c->wl = wl;
   c->n_sm = n_sm;
+  c->per_seq = cfg->per_sequence_budgets != 0;
   c->begun = false;
   c->budget_state = 0;
-  c->hs = nullptr;
-  if (cudaHostAlloc(reinterpret_cast<void**>(&c->hs), sizeof(HostStage), cudaHostAllocDefault) != cudaSuccess ||
+  // one pinned block, carved into the staging arrays (largest alignment first)
+  const size_t nd = wl.n_desc_cap;
+  const size_t bytes = nd * (sizeof(LayerDesc) + sizeof(EvictLayer) + 8 + 4 + 4 + 4 + 4 + 1) + 64;
+  void* blk = nullptr;
+  if (cudaHostAlloc(&blk, bytes, cudaHostAllocDefault) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev, cudaEventDisableTiming) != cudaSuccess) {
-    if (c->hs) cudaFreeHost(c->hs);
+    if (blk) cudaFreeHost(blk);
     delete c;
     return SQ_ERR_CUDA;
   }
-  std::memset(c->hs, 0, sizeof(HostStage));
+  std::memset(blk, 0, bytes);
+  char* p = static_cast<char*>(blk);
+  c->hs.block = blk;
+  c->hs.layers = reinterpret_cast<LayerDesc*>(p);
+  p += nd * sizeof(LayerDesc);
+  c->hs.evict_tab = reinterpret_cast<EvictLayer*>(p);
+  p += nd * sizeof(EvictLayer);
+  c->hs.tok_count = reinterpret_cast<long long*>(p);
+  p += nd * 8;
+  c->hs.budget = reinterpret_cast<int32_t*>(p);
+  p += nd * 4;
+  c->hs.cos_sim = reinterpret_cast<float*>(p);
+  p += nd * 4;
+  c->hs.order = reinterpret_cast<int*>(p);
+  p += nd * 4;
+  c->hs.order_by_layer = reinterpret_cast<int*>(p);
+  p += nd * 4;
+  c->hs.is_g3 = reinterpret_cast<uint8_t*>(p);
   *out = c;
   return SQ_OK;
 }
@@ -254,7 +307,7 @@ int sq_ctx_create(const sq_config* cfg, int64_t b_init, void* pool, size_t pool_
 int sq_ctx_destroy(sq_ctx* c) {
   if (!c) return SQ_ERR_INVALID_ARG;
   cudaEventDestroy(c->ev);
-  cudaFreeHost(c->hs);
+  cudaFreeHost(c->hs.block);
   delete c;
   return SQ_OK;
 }
@@ -268,14 +321,18 @@ int sq_begin_sequence_batch(sq_ctx* c, int32_t batch, int32_t prompt_len, void* 
   if (prompt_len < 1 || prompt_len > c->cfg.max_prompt) return fail(c, SQ_ERR_INVALID_ARG, "prompt_len out of range");
   c->batch = batch;
   c->prompt = prompt_len;
+  c->n_grp = c->per_seq ? batch : 1;
+  c->desc_units = c->per_seq ? c->cfg.n_kv_head : batch * c->cfg.n_kv_head;
+  c->n_desc = c->cfg.n_layer * c->n_grp;
   c->begun = true;
   c->budget_state = 0;
   for (int l = 0; l < c->cfg.n_layer; ++l) {
     c->n_tok[l] = 0;
+    c->imp_tokens[l] = 0;
     c->prefilled[l] = false;
     c->importance_seen[l] = false;
-    c->hs->tok_count[l] = 0;
   }
+  for (int d = 0; d < c->n_desc; ++d) c->hs.tok_count[d] = 0;
   // everything up to the layer table: statistics, ticket, budgets, status
   SQ_CUDA(c, cudaMemsetAsync(c->ws, 0, c->wl.layers, st));
   return SQ_OK;
@@ -290,18 +347,36 @@ int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const v
     return fail(c, SQ_ERR_INVALID_ARG, "hidden state pointers must be non-NULL and 16-byte aligned");
   if (n_tok_total < 0) return fail(c, SQ_ERR_INVALID_ARG, "n_tok_total is negative");
   if (n_tok_total == 0) return SQ_OK;
-  ImportanceArgs a;
-  a.a = hidden_in;
-  a.b = hidden_out;
-  a.n_tok = n_tok_total;
-  a.hidden = c->cfg.hidden;
-  a.cta_partial = ws_ptr<float>(c, c->wl.cta_partial);
-  a.ticket = ws_ptr<unsigned int>(c, c->wl.ticket);
-  a.cos_sum = ws_ptr<double>(c, c->wl.cos_sum) + layer;
-  long long want = (n_tok_total + 7) / 8;
-  int n_cta = (int)std::min<long long>(want, std::min(kMaxImportanceCtas, c->n_sm * 8));
-  SQ_CUDA(c, launch_importance(a, c->cfg.dtype, n_cta, static_cast<cudaStream_t>(stream)));
-  c->hs->tok_count[layer] += n_tok_total;
+  if (c->per_seq && c->imp_tokens[layer] + n_tok_total > (long long)c->batch * c->prompt)
+    return fail(c, SQ_ERR_INVALID_ARG, "more tokens than batch * prompt_len for this layer");
+  const size_t row = (size_t)c->cfg.hidden * elem_bytes(c->cfg.dtype);
+  long long done = 0;
+  while (done < n_tok_total) {
+    // with per-sequence budgets the rows are taken sequence by sequence, prompt_len rows each:
+    // a call is cut at the sequence boundaries it spans
+    long long n = n_tok_total - done;
+    int grp = 0;
+    if (c->per_seq) {
+      const long long t = c->imp_tokens[layer] + done;
+      grp = (int)(t / c->prompt);
+      n = std::min<long long>(n, (long long)(grp + 1) * c->prompt - t);
+    }
+    const int d = layer * c->n_grp + grp;
+    ImportanceArgs a;
+    a.a = static_cast<const char*>(hidden_in) + (size_t)done * row;
+    a.b = static_cast<const char*>(hidden_out) + (size_t)done * row;
+    a.n_tok = n;
+    a.hidden = c->cfg.hidden;
+    a.cta_partial = ws_ptr<float>(c, c->wl.cta_partial);
+    a.ticket = ws_ptr<unsigned int>(c, c->wl.ticket);
+    a.cos_sum = ws_ptr<double>(c, c->wl.cos_sum) + d;
+    long long want = (n + 7) / 8;
+    int n_cta = (int)std::min<long long>(want, std::min(kMaxImportanceCtas, c->n_sm * 8));
+    SQ_CUDA(c, launch_importance(a, c->cfg.dtype, n_cta, static_cast<cudaStream_t>(stream)));
+    c->hs.tok_count[d] += n;
+    done += n;
+  }
+  c->imp_tokens[layer] += n_tok_total;
   c->importance_seen[layer] = true;
   return SQ_OK;
 }
@@ -312,24 +387,28 @@ int sq_allocate_budgets(sq_ctx* c, int64_t b_init, double p, void* stream) {
   if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
   if (!(p > 0.0 && p <= 1.0)) return fail(c, SQ_ERR_INVALID_ARG, "p must satisfy 0 < p <= 1");
   if (b_init < 1 || b_init > c->b_init_cap) return fail(c, SQ_ERR_INVALID_ARG, "b_init must be in 1..the context's b_init");
-  for (int l = 0; l < c->cfg.n_layer; ++l)
+  for (int l = 0; l < c->cfg.n_layer; ++l) {
     if (!c->importance_seen[l]) return fail(c, SQ_ERR_STATE, "sq_layer_importance has not been called for every layer");
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<long long>(c, c->wl.tok_count), c->hs->tok_count, 8 * c->cfg.n_layer,
-                             cudaMemcpyHostToDevice, st));
+    if (c->per_seq && c->imp_tokens[l] != (long long)c->batch * c->prompt)
+      return fail(c, SQ_ERR_STATE, "per-sequence budgets need the hidden states of every prompt token of every layer");
+  }
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<long long>(c, c->wl.tok_count), c->hs.tok_count, 8 * c->n_desc, cudaMemcpyHostToDevice,
+                             st));
   AllocateArgs a;
   a.cos_sum = ws_ptr<double>(c, c->wl.cos_sum);
   a.tok_count = ws_ptr<long long>(c, c->wl.tok_count);
   a.n_layer = c->cfg.n_layer;
   a.n_cluster = c->cfg.n_cluster;
+  a.stride = c->n_grp;
   a.b_init = b_init;
   a.p = p;
   a.cos_sim = ws_ptr<float>(c, c->wl.cos_sim);
   a.budget = ws_ptr<int>(c, c->wl.budget);
   a.is_g3 = ws_ptr<unsigned char>(c, c->wl.is_g3);
   SQ_CUDA(c, launch_allocate(a, st));
-  SQ_CUDA(c, cudaMemcpyAsync(c->hs->budget, a.budget, 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
-  SQ_CUDA(c, cudaMemcpyAsync(c->hs->is_g3, a.is_g3, c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
-  SQ_CUDA(c, cudaMemcpyAsync(c->hs->cos_sim, a.cos_sim, 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs.budget, a.budget, 4 * c->n_desc, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs.is_g3, a.is_g3, c->n_desc, cudaMemcpyDeviceToHost, st));
+  SQ_CUDA(c, cudaMemcpyAsync(c->hs.cos_sim, a.cos_sim, 4 * c->n_desc, cudaMemcpyDeviceToHost, st));
   SQ_CUDA(c, cudaEventRecord(c->ev, st));
   c->budget_state = 1;
   for (int l = 0; l < c->cfg.n_layer; ++l) c->prefilled[l] = false;
@@ -343,12 +422,14 @@ int sq_set_budgets(sq_ctx* c, const int32_t* budgets_host, void* stream) {
   if (!budgets_host) return fail(c, SQ_ERR_INVALID_ARG, "budgets_host is NULL");
   if (c->budget_state == 1) SQ_CUDA(c, cudaEventSynchronize(c->ev));
   for (int l = 0; l < c->cfg.n_layer; ++l) {
-    c->hs->budget[l] = budgets_host[l];
-    c->hs->is_g3[l] = 0;
+    for (int g = 0; g < c->n_grp; ++g) {
+      c->hs.budget[l * c->n_grp + g] = budgets_host[user_index(c, l, g)];
+      c->hs.is_g3[l * c->n_grp + g] = 0;
+    }
     c->prefilled[l] = false;
   }
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs->budget, 4 * c->cfg.n_layer, cudaMemcpyHostToDevice, st));
-  SQ_CUDA(c, cudaMemsetAsync(ws_ptr<unsigned char>(c, c->wl.is_g3), 0, c->cfg.n_layer, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs.budget, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemsetAsync(ws_ptr<unsigned char>(c, c->wl.is_g3), 0, c->n_desc, st));
   c->budget_state = 0;
   int rc = build_layout(c, st);
   return rc;
@@ -366,14 +447,13 @@ int sq_prefill_compress(sq_ctx* c, int32_t layer, const void* k_prompt, const vo
   if (h2o && !q_prompt && !acc_prompt) return fail(c, SQ_ERR_INVALID_ARG, "H2O needs q_prompt or acc_prompt");
   int rc = ensure_budgets(c, st);
   if (rc != SQ_OK) return rc;
-  const LayerDesc& ld = c->hs->layers[layer];
-  const int U = c->batch * c->cfg.n_kv_head, P = c->prompt;
-  const int n_keep = std::min(P, ld.b);
+  const int P = c->prompt, U = c->desc_units;
   const float* acc = nullptr;
   if (h2o) {
     if (acc_prompt) {
       acc = acc_prompt;
     } else {
+      // the scores do not depend on the budgets: one pass for the whole batch
       ScoreArgs s;
       s.q = q_prompt;
       s.k = k_prompt;
@@ -387,21 +467,28 @@ int sq_prefill_compress(sq_ctx* c, int32_t layer, const void* k_prompt, const vo
       SQ_CUDA(c, launch_prefill_scores(s, c->cfg.dtype, ws_ptr<int>(c, c->wl.status), st));
       acc = s.acc_prompt;
     }
-    SQ_CUDA(c, launch_select_prompt(acc, U, P, ld, c->pool, st));
   }
-  GatherArgs g;
-  g.k_prompt = k_prompt;
-  g.v_prompt = v_prompt;
-  g.acc_prompt = acc;
-  g.pool = c->pool;
-  g.ld = ld;
-  g.n_unit = U;
-  g.prompt = P;
-  g.n_keep = n_keep;
-  g.policy = c->cfg.policy;
-  g.head_dim = c->cfg.head_dim;
-  SQ_CUDA(c, launch_gather(g, c->cfg.dtype, st));
-  if (h2o && n_keep == ld.b) SQ_CUDA(c, launch_pick_victim(c->pool, ld, U, n_keep, P, st));
+  // selection and gather per descriptor (the whole batch, or one sequence at a time)
+  const size_t kv_stride = (size_t)U * P * c->cfg.head_dim * elem_bytes(c->cfg.dtype);
+  for (int g = 0; g < c->n_grp; ++g) {
+    const LayerDesc& ld = c->hs.layers[layer * c->n_grp + g];
+    const int n_keep = std::min(P, ld.b);
+    const float* acc_g = acc ? acc + (size_t)g * U * P : nullptr;
+    if (h2o) SQ_CUDA(c, launch_select_prompt(acc_g, U, P, ld, c->pool, st));
+    GatherArgs ga;
+    ga.k_prompt = static_cast<const char*>(k_prompt) + g * kv_stride;
+    ga.v_prompt = static_cast<const char*>(v_prompt) + g * kv_stride;
+    ga.acc_prompt = acc_g;
+    ga.pool = c->pool;
+    ga.ld = ld;
+    ga.n_unit = U;
+    ga.prompt = P;
+    ga.n_keep = n_keep;
+    ga.policy = c->cfg.policy;
+    ga.head_dim = c->cfg.head_dim;
+    SQ_CUDA(c, launch_gather(ga, c->cfg.dtype, st));
+    if (h2o && n_keep == ld.b) SQ_CUDA(c, launch_pick_victim(c->pool, ld, U, n_keep, P, st));
+  }
   c->n_tok[layer] = P;
   c->prefilled[layer] = true;
   return SQ_OK;
@@ -423,7 +510,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     if (!c->prefilled[l]) return fail(c, SQ_ERR_STATE, "sq_prefill_compress has not been called for a layer in the range");
     if (c->n_tok[l] >= cfg.max_prompt + cfg.max_new_tokens) return fail(c, SQ_ERR_CAPACITY, "max_new_tokens exceeded");
   }
-  const int U = c->batch * cfg.n_kv_head, G = cfg.n_q_head / cfg.n_kv_head;
+  const int U = c->desc_units, G = cfg.n_q_head / cfg.n_kv_head, ng = c->n_grp;
   const size_t eb = elem_bytes(cfg.dtype);
   const size_t q_layer = (size_t)c->batch * cfg.n_q_head * cfg.head_dim * eb;
   const size_t kv_layer = (size_t)c->batch * cfg.n_kv_head * cfg.head_dim * eb;
@@ -432,11 +519,13 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     int e = s + 1;
     while (e < layer_end && c->n_tok[e] == c->n_tok[s]) ++e;
     const int n_tok = c->n_tok[s];
+    const int d0 = s * ng, d1 = e * ng;  // descriptors of the launch
     // Split-K plan.  A piece costs a fixed set-up plus its tiles, and pieces run in waves of
     // as many CTAs as fit the GPU at once; among the piece lengths that are whole tiles, take
     // the one with the smallest estimated time.  What a tile, a set-up (in tiles; fitted to
     // measured step times, it includes writing and merging the partial results) and a wave are
-    // depends on the kernel the shape is served by.
+    // depends on the kernel the shape is served by.  With per-sequence budgets the units of a
+    // layer differ in length and are not split: every descriptor has exactly U items.
     const bool bf16 = cfg.dtype == SQ_BF16;
     int tile, setup, per_sm;
     if (bf16 && cfg.head_dim == 64 && G > 32) {  // tcgen05 kernel: 128-token tiles, 2 CTAs per SM
@@ -448,22 +537,22 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     }
     const long long slots = (long long)per_sm * c->n_sm;
     int max_len = 1;
-    for (int l = s; l < e; ++l) max_len = std::max(max_len, std::min(n_tok + 1, c->hs->layers[l].b));
+    for (int d = d0; d < d1; ++d) max_len = std::max(max_len, std::min(n_tok + 1, c->hs.layers[d].b));
     int split = 0;
     double best_cost = 0.0;
     int prev = -1;
     static const int forced = [] {  // SQ_SPLIT_PIECES=n forces n pieces per longest unit (for measurements)
-      const char* e = getenv("SQ_SPLIT_PIECES");
-      return e ? atoi(e) : 0;
+      const char* ev = getenv("SQ_SPLIT_PIECES");
+      return ev ? atoi(ev) : 0;
     }();
-    for (int pieces = 1; pieces <= 64; ++pieces) {
+    for (int pieces = 1; pieces <= (c->per_seq ? 1 : 64); ++pieces) {
       int cand = ((max_len + pieces - 1) / pieces + tile - 1) / tile * tile;
       if (pieces > 1 && cand < 2 * tile) break;  // a piece is never shorter than two tiles
       if (cand == prev) continue;
       prev = cand;
       long long items = 0, work = 0;
-      for (int l = s; l < e; ++l) {
-        const int len = std::min(n_tok + 1, c->hs->layers[l].b);
+      for (int d = d0; d < d1; ++d) {
+        const int len = std::min(n_tok + 1, c->hs.layers[d].b);
         const int ns = (len + cand - 1) / cand;
         items += (long long)U * ns;
         work += (long long)U * ((long long)ns * setup + (len + tile - 1) / tile);
@@ -481,15 +570,14 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
       }
     }
     long long n_items = 0;
-    for (int l = s; l < e; ++l) {
-      int len = std::min(n_tok + 1, c->hs->layers[l].b);
+    for (int d = d0; d < d1; ++d) {
+      int len = std::min(n_tok + 1, c->hs.layers[d].b);
       int ns = (len + split - 1) / split;
       n_items += (long long)U * ns;
     }
     if ((size_t)n_items > c->wl.items_cap) return fail(c, SQ_ERR_CAPACITY, "workspace too small for the split plan");
     DecodeArgs a;
     a.layers = ws_ptr<LayerDesc>(c, c->wl.layers);
-    a.order = ws_ptr<int>(c, c->wl.order);
     a.pool = c->pool;
     a.logits = ws_ptr<float>(c, c->wl.logits);
     a.part_stat = ws_ptr<float>(c, c->wl.part_stat);
@@ -500,11 +588,20 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.out = static_cast<char*>(out) + (size_t)(s - layer_begin) * q_layer;
     a.status = ws_ptr<int>(c, c->wl.status);
     a.tickets = ws_ptr<int>(c, c->wl.tickets);
-    a.n_layer_total = cfg.n_layer;
-    a.layer_begin = s;
-    a.layer_end = e;
+    a.uniform = c->per_seq ? 1 : 0;
+    if (c->per_seq) {
+      // the launch's descriptors only: the global order for the whole stack, else layer by layer
+      const bool all = (s == 0 && e == cfg.n_layer);
+      a.order = all ? ws_ptr<int>(c, c->wl.order) : ws_ptr<int>(c, c->wl.order_by_layer) + d0;
+      a.n_layer_total = d1 - d0;
+    } else {
+      a.order = ws_ptr<int>(c, c->wl.order);
+      a.n_layer_total = c->n_desc;
+    }
+    a.layer_begin = d0;
+    a.layer_end = d1;
     a.n_tok = n_tok;
-    a.batch = c->batch;
+    a.batch = c->per_seq ? 1 : c->batch;
     a.n_q_head = cfg.n_q_head;
     a.n_kv_head = cfg.n_kv_head;
     a.head_dim = cfg.head_dim;
@@ -531,73 +628,79 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
   int rc = ensure_budgets(c, st);
   if (rc != SQ_OK) return rc;
   const sq_config& cfg = c->cfg;
+  const int ng = c->n_grp, nl = layer_end - layer_begin;
+  // new_budgets_host: [layer_end - layer_begin], or [batch][layer_end - layer_begin] with per-sequence budgets
+  auto new_budget = [&](int l, int g) { return new_budgets_host[g * nl + (l - layer_begin)]; };
   for (int l = layer_begin; l < layer_end; ++l) {
-    const int nb = new_budgets_host[l - layer_begin];
     if (!c->prefilled[l]) return fail(c, SQ_ERR_STATE, "sq_prefill_compress has not been called for a layer in the range");
-    if (nb < 1 || nb > c->hs->layers[l].b) return fail(c, SQ_ERR_INVALID_ARG, "new budget must be in 1..current budget");
-    if (cfg.policy == SQ_POLICY_STREAMING_LLM && nb <= cfg.n_sink)
-      return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
+    for (int g = 0; g < ng; ++g) {
+      const int nb = new_budget(l, g);
+      if (nb < 1 || nb > c->hs.layers[l * ng + g].b) return fail(c, SQ_ERR_INVALID_ARG, "new budget must be in 1..current budget");
+      if (cfg.policy == SQ_POLICY_STREAMING_LLM && nb <= cfg.n_sink)
+        return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
+    }
   }
-  const int U = c->batch * cfg.n_kv_head;
   int n_active = 0, max_cap = 0;
   for (int l = layer_begin; l < layer_end; ++l) {
-    const int nb = new_budgets_host[l - layer_begin];
-    LayerDesc old = c->hs->layers[l];
-    if (nb == old.b) continue;
-    LayerDesc nw = old;
-    nw.b = nb;
-    nw.b_heavy = cfg.policy == SQ_POLICY_H2O ? (int)(((long long)nb * cfg.heavy_num) / cfg.heavy_den) : 0;
-    nw.b_recent = nb - nw.b_heavy;
-    const int n_tok = c->n_tok[l];
-    const int len = std::min(n_tok, old.b);
-    if (cfg.policy != SQ_POLICY_H2O) {
-      // the compaction keeps slot order, so the ring stays a rotation: find its new phase
-      const int base = old.ring_base, r_old = old.b - base, r_new = nb - base;
-      if (n_tok <= nb) {
-        nw.ring_origin = base;
-      } else {
-        const int x0 = n_tok - r_new;
-        const int r0 = (x0 - old.ring_origin) % r_old;
-        const int h = (r0 + r_new <= r_old) ? 0 : r0 + r_new - r_old;
-        nw.ring_origin = x0 - h;
+    for (int g = 0; g < ng; ++g) {
+      const int d = l * ng + g;
+      const int nb = new_budget(l, g);
+      LayerDesc old = c->hs.layers[d];
+      if (nb == old.b) continue;
+      LayerDesc nw = old;
+      nw.b = nb;
+      nw.b_heavy = cfg.policy == SQ_POLICY_H2O ? (int)(((long long)nb * cfg.heavy_num) / cfg.heavy_den) : 0;
+      nw.b_recent = nb - nw.b_heavy;
+      const int n_tok = c->n_tok[l];
+      const int len = std::min(n_tok, old.b);
+      if (cfg.policy != SQ_POLICY_H2O) {
+        // the compaction keeps slot order, so the ring stays a rotation: find its new phase
+        const int base = old.ring_base, r_old = old.b - base, r_new = nb - base;
+        if (n_tok <= nb) {
+          nw.ring_origin = base;
+        } else {
+          const int x0 = n_tok - r_new;
+          const int r0 = (x0 - old.ring_origin) % r_old;
+          const int h = (r0 + r_new <= r_old) ? 0 : r0 + r_new - r_old;
+          nw.ring_origin = x0 - h;
+        }
       }
+      if (len > nb) {
+        EvictLayer& ev = c->hs.evict_tab[n_active++];
+        ev.ld_old = old;
+        ev.ld_new = nw;
+        ev.len = len;
+        ev.n_tok = n_tok;
+        max_cap = std::max(max_cap, old.cap);
+      }
+      c->hs.layers[d] = nw;
+      c->hs.budget[d] = nb;
     }
-    if (len > nb) {
-      EvictLayer& e = c->hs->evict_tab[n_active++];
-      e.ld_old = old;
-      e.ld_new = nw;
-      e.len = len;
-      e.n_tok = n_tok;
-      max_cap = std::max(max_cap, old.cap);
-    }
-    c->hs->layers[l] = nw;
-    c->hs->budget[l] = nb;
   }
   if (n_active > 0) {
-    // all layers of the call in one launch
+    // all descriptors of the call in one launch
     EvictArgs a;
     a.pool = c->pool;
     a.tab = ws_ptr<EvictLayer>(c, c->wl.evict_tab);
     a.n_layers = n_active;
     a.max_cap = max_cap;
-    a.n_unit = U;
+    a.n_unit = c->desc_units;
     a.policy = cfg.policy;
     a.n_sink = cfg.n_sink;
     a.row_bytes = cfg.head_dim * elem_bytes(cfg.dtype);
     a.status = ws_ptr<int>(c, c->wl.status);
-    SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<EvictLayer>(c, c->wl.evict_tab), c->hs->evict_tab, sizeof(EvictLayer) * n_active,
+    SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<EvictLayer>(c, c->wl.evict_tab), c->hs.evict_tab, sizeof(EvictLayer) * n_active,
                                cudaMemcpyHostToDevice, st));
     SQ_CUDA(c, launch_evict(a, st));
   }
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers) + layer_begin, &c->hs->layers[layer_begin],
-                             sizeof(LayerDesc) * (layer_end - layer_begin), cudaMemcpyHostToDevice, st));
-  // the launch order (largest budget first) may have changed
-  std::vector<int> ord(cfg.n_layer);
-  for (int l = 0; l < cfg.n_layer; ++l) ord[l] = l;
-  std::stable_sort(ord.begin(), ord.end(), [&](int x, int y) { return c->hs->budget[x] > c->hs->budget[y]; });
-  std::copy(ord.begin(), ord.end(), c->hs->order);
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs->order, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
-  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs->budget, 4 * cfg.n_layer, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers) + layer_begin * ng, &c->hs.layers[layer_begin * ng],
+                             sizeof(LayerDesc) * nl * ng, cudaMemcpyHostToDevice, st));
+  // the launch orders (largest budget first) may have changed
+  sort_orders(c);
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs.order, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order_by_layer), c->hs.order_by_layer, 4 * c->n_desc,
+                             cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs.budget, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
   SQ_CUDA(c, cudaStreamSynchronize(st));
   return SQ_OK;
 }
@@ -606,7 +709,10 @@ int sq_get_cos_sim(sq_ctx* c, float* cos_sim_host) {
   if (!c || !cos_sim_host) return SQ_ERR_INVALID_ARG;
   if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "sq_allocate_budgets has not been called");
   SQ_CUDA(c, cudaDeviceSynchronize());
-  SQ_CUDA(c, cudaMemcpy(cos_sim_host, ws_ptr<float>(c, c->wl.cos_sim), 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  std::vector<float> tmp(c->n_desc);
+  SQ_CUDA(c, cudaMemcpy(tmp.data(), ws_ptr<float>(c, c->wl.cos_sim), 4 * c->n_desc, cudaMemcpyDeviceToHost));
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    for (int g = 0; g < c->n_grp; ++g) cos_sim_host[user_index(c, l, g)] = tmp[l * c->n_grp + g];
   return SQ_OK;
 }
 
@@ -614,10 +720,22 @@ int sq_get_budgets(sq_ctx* c, int32_t* budgets_host, uint8_t* is_g3_host) {
   if (!c || !budgets_host) return SQ_ERR_INVALID_ARG;
   if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "budgets not set");
   SQ_CUDA(c, cudaDeviceSynchronize());
-  SQ_CUDA(c, cudaMemcpy(budgets_host, ws_ptr<int>(c, c->wl.budget), 4 * c->cfg.n_layer, cudaMemcpyDeviceToHost));
-  if (is_g3_host)
-    SQ_CUDA(c, cudaMemcpy(is_g3_host, ws_ptr<unsigned char>(c, c->wl.is_g3), c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  std::vector<int32_t> tb(c->n_desc);
+  std::vector<uint8_t> tg(c->n_desc);
+  SQ_CUDA(c, cudaMemcpy(tb.data(), ws_ptr<int>(c, c->wl.budget), 4 * c->n_desc, cudaMemcpyDeviceToHost));
+  SQ_CUDA(c, cudaMemcpy(tg.data(), ws_ptr<unsigned char>(c, c->wl.is_g3), c->n_desc, cudaMemcpyDeviceToHost));
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    for (int g = 0; g < c->n_grp; ++g) {
+      budgets_host[user_index(c, l, g)] = tb[l * c->n_grp + g];
+      if (is_g3_host) is_g3_host[user_index(c, l, g)] = tg[l * c->n_grp + g];
+    }
   return SQ_OK;
+}
+
+// Where a unit lives: its descriptor and its index within it.
+static const LayerDesc& unit_desc(sq_ctx* c, int layer, int seq, int kv_head, size_t* unit) {
+  *unit = c->per_seq ? (size_t)kv_head : (size_t)seq * c->cfg.n_kv_head + kv_head;
+  return c->hs.layers[layer * c->n_grp + (c->per_seq ? seq : 0)];
 }
 
 static int unit_order(sq_ctx* c, int layer, int seq, int kv_head, std::vector<int>& pos, std::vector<int>& order) {
@@ -625,9 +743,9 @@ static int unit_order(sq_ctx* c, int layer, int seq, int kv_head, std::vector<in
     return fail(c, SQ_ERR_INVALID_ARG, "layer/seq/kv_head out of range");
   if (c->budget_state != 2 || !c->prefilled[layer]) return fail(c, SQ_ERR_STATE, "layer has no cache yet");
   SQ_CUDA(c, cudaDeviceSynchronize());
-  const LayerDesc& ld = c->hs->layers[layer];
+  size_t unit;
+  const LayerDesc& ld = unit_desc(c, layer, seq, kv_head, &unit);
   const int len = std::min(c->n_tok[layer], ld.b);
-  const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
   pos.resize(len);
   SQ_CUDA(c, cudaMemcpy(pos.data(), c->pool + ld.pos_off + unit * ld.cap * 4, (size_t)len * 4, cudaMemcpyDeviceToHost));
   order.resize(len);
@@ -641,13 +759,12 @@ int sq_get_kept(sq_ctx* c, int32_t layer, int32_t seq, int32_t kv_head, int32_t*
   std::vector<int> pos, order;
   int rc = unit_order(c, layer, seq, kv_head, pos, order);
   if (rc != SQ_OK) return rc;
-  const LayerDesc& ld = c->hs->layers[layer];
+  size_t unit;
+  const LayerDesc& ld = unit_desc(c, layer, seq, kv_head, &unit);
   const int len = (int)pos.size();
   std::vector<float> acc(len, 0.f);
-  if (c->cfg.policy == SQ_POLICY_H2O && len > 0) {
-    const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
+  if (c->cfg.policy == SQ_POLICY_H2O && len > 0)
     SQ_CUDA(c, cudaMemcpy(acc.data(), c->pool + ld.acc_off + unit * ld.cap * 4, (size_t)len * 4, cudaMemcpyDeviceToHost));
-  }
   for (int i = 0; i < len; ++i) {
     pos_host[i] = pos[order[i]];
     if (acc_host) acc_host[i] = acc[order[i]];
@@ -661,10 +778,10 @@ int sq_get_kv(sq_ctx* c, int32_t layer, int32_t seq, int32_t kv_head, void* k_ho
   std::vector<int> pos, order;
   int rc = unit_order(c, layer, seq, kv_head, pos, order);
   if (rc != SQ_OK) return rc;
-  const LayerDesc& ld = c->hs->layers[layer];
+  size_t unit;
+  const LayerDesc& ld = unit_desc(c, layer, seq, kv_head, &unit);
   const int len = (int)pos.size();
   const size_t row = (size_t)c->cfg.head_dim * elem_bytes(c->cfg.dtype);
-  const size_t unit = (size_t)seq * c->cfg.n_kv_head + kv_head;
   std::vector<char> kb(len * row), vb(len * row);
   if (len > 0) {
     SQ_CUDA(c, cudaMemcpy(kb.data(), c->pool + ld.k_off + unit * ld.cap * row, len * row, cudaMemcpyDeviceToHost));
@@ -681,7 +798,9 @@ int sq_get_len(sq_ctx* c, int32_t layer, int32_t* len) {
   if (!c || !len) return SQ_ERR_INVALID_ARG;
   if (layer < 0 || layer >= c->cfg.n_layer) return fail(c, SQ_ERR_INVALID_ARG, "layer out of range");
   if (c->budget_state != 2 || !c->prefilled[layer]) return fail(c, SQ_ERR_STATE, "layer has no cache yet");
-  *len = std::min(c->n_tok[layer], c->hs->layers[layer].b);
+  int longest = 0;  // with per-sequence budgets: the longest of the layer's sequences
+  for (int g = 0; g < c->n_grp; ++g) longest = std::max(longest, std::min(c->n_tok[layer], c->hs.layers[layer * c->n_grp + g].b));
+  *len = longest;
   return SQ_OK;
 }
 
@@ -697,11 +816,12 @@ int sq_kv_bytes_per_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, int6
   if (layer_begin < 0 || layer_end > c->cfg.n_layer || layer_begin >= layer_end)
     return fail(c, SQ_ERR_INVALID_ARG, "layer range");
   if (c->budget_state != 2) return fail(c, SQ_ERR_STATE, "budgets not on the host yet");
-  const int64_t U = (int64_t)c->batch * c->cfg.n_kv_head;
+  const int64_t U = c->desc_units;
   const int64_t row = (int64_t)c->cfg.head_dim * elem_bytes(c->cfg.dtype);
   int64_t total = 0;
   for (int l = layer_begin; l < layer_end; ++l)
-    total += U * std::min(c->n_tok[l] + 1, c->hs->layers[l].b) * 2 * row;
+    for (int g = 0; g < c->n_grp; ++g)
+      total += U * std::min(c->n_tok[l] + 1, c->hs.layers[l * c->n_grp + g].b) * 2 * row;
   *bytes = total;
   return SQ_OK;
 }

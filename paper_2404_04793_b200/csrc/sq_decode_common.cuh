@@ -24,6 +24,15 @@ __device__ __forceinline__ int n_split_of(const DecodeArgs& a, int b) {
 // layers, either the layer an item index falls in (want_layer < 0) or the first item of a
 // given layer.
 __device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_layer, ItemLoc& out) {
+  if (a.uniform) {  // `order` lists exactly the launch's descriptors, n_unit items each
+    const int k = idx / a.n_unit;
+    if (k >= a.n_layer_total) return false;
+    out.layer = a.order[k];
+    out.n_split = 1;
+    out.base = k * a.n_unit;
+    out.local = idx - out.base;
+    return true;
+  }
   const int lane = threadIdx.x & 31;
   int running = 0;
   for (int c = 0; c < a.n_layer_total; c += 32) {

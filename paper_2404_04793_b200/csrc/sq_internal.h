@@ -40,10 +40,10 @@ struct ImportanceArgs {
   double* cos_sum;       // += sum over tokens of the cosine
 };
 
-struct AllocateArgs {
+struct AllocateArgs {  // entry of layer i: [i * stride + blockIdx.x] (one CTA per budget vector)
   const double* cos_sum;
   const long long* tok_count;
-  int n_layer, n_cluster;
+  int n_layer, n_cluster, stride;
   long long b_init;
   double p;
   float* cos_sim;
@@ -68,9 +68,11 @@ struct ScoreArgs {  // H2O prompt scores of one layer
   int batch, n_q_head, n_kv_head, prompt, head_dim;
 };
 
+// "Layer" below means one cache descriptor: a layer of the whole batch, or, with per-sequence
+// budgets, a (layer, sequence) pair holding that sequence's n_kv_head units (batch = 1 then).
 struct DecodeArgs {
   const LayerDesc* layers;
-  const int* order;  // layer indices sorted by budget, descending
+  const int* order;  // descriptor indices sorted by budget, descending; with `uniform` only those of the launch
   char* pool;
   float* logits;
   float* part_stat;  // [item][group][4]   (max, sum, sum of rounded weights, pad) in the log2 domain
@@ -86,6 +88,7 @@ struct DecodeArgs {
   int batch, n_q_head, n_kv_head, head_dim, group;
   int n_unit;  // batch * n_kv_head
   int split_tokens, policy;
+  int uniform;  // every descriptor of the launch has n_unit items (no split-K): items are found in O(1)
   float scale_log2;  // log2(e) / sqrt(head_dim)
 };
 
