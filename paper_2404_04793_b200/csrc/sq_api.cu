@@ -588,8 +588,9 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.out = static_cast<char*>(out) + (size_t)(s - layer_begin) * q_layer;
     a.status = ws_ptr<int>(c, c->wl.status);
     a.tickets = ws_ptr<int>(c, c->wl.tickets);
-    a.uniform = c->per_seq ? 1 : 0;
-    if (c->per_seq) {
+    // without split-K every descriptor has exactly U items and an item is found in O(1)
+    a.uniform = (n_items == (long long)U * (d1 - d0)) ? 1 : 0;
+    if (a.uniform) {
       // the launch's descriptors only: the global order for the whole stack, else layer by layer
       const bool all = (s == 0 && e == cfg.n_layer);
       a.order = all ? ws_ptr<int>(c, c->wl.order) : ws_ptr<int>(c, c->wl.order_by_layer) + d0;

@@ -40,7 +40,7 @@ def build_workload(args) -> synth.Workload:
     return w
 
 
-def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, device="cuda:0"):
+def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, device="cuda:0", per_sequence=False):
     job = engine.Job(w.replace(steps=steps + warmup), device)
     ctx = job.ctx
     ctx.begin_sequence_batch(w.batch, w.prompt)
@@ -49,6 +49,15 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
         ctx.layer_importance(l, a, b)
     ctx.allocate_budgets(w.b_init, w.p)
     budgets, _ = ctx.get_budgets()
+    if per_sequence:
+        # same budget vector rotated by one layer per sequence: every sequence has its own
+        # budgets (equal totals), as the per-sequence allocation would produce on unlike prompts
+        ctx.close()
+        ctx = job.ctx = engine.context_for(job.w, device, per_sequence_budgets=1)
+        ctx.begin_sequence_batch(w.batch, w.prompt)
+        rows = [budgets[s % w.n_layer:] + budgets[:s % w.n_layer] for s in range(w.batch)]
+        ctx.set_budgets(rows)
+        budgets = [sum(r[l] for r in rows) / w.batch for l in range(w.n_layer)]   # mean per layer, for the byte count
     g = torch.Generator(device=device).manual_seed(1)
     shape_kv = (w.batch, w.n_kv_head, w.prompt, w.head_dim)
     k = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
@@ -93,13 +102,13 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     e = 2 if w.dtype == torch.bfloat16 else 4
-    kv = w.batch * w.n_kv_head * sum(min(w.prompt + 1, b) for b in budgets) * 2 * w.head_dim * e
+    kv = int(w.batch * w.n_kv_head * sum(min(w.prompt + 1, b) for b in budgets) * 2 * w.head_dim * e)
     io = w.batch * w.n_layer * (2 * w.n_q_head + 2 * w.n_kv_head) * w.head_dim * e
-    extra = (w.batch * w.n_kv_head * sum(budgets) * 8) if w.policy == synth.H2O else 0
+    extra = int(w.batch * w.n_kv_head * sum(budgets) * 8) if w.policy == synth.H2O else 0
     gbs = (kv + io + extra) / ms / 1e6
-    return dict(workload=w.name, per_layer=per_layer, ms_per_step=round(ms, 4), GBs=round(gbs, 1),
+    return dict(workload=w.name, per_layer=per_layer, per_sequence_budgets=per_sequence, ms_per_step=round(ms, 4), GBs=round(gbs, 1),
                 kv_GB=round(kv / 1e9, 3), algorithmic_bytes=kv + io + extra, tokens_per_s=round(w.batch / ms * 1e3),
-                flops=4 * w.n_q_head * w.head_dim * w.batch * sum(budgets), device_status=ctx.status())
+                flops=int(4 * w.n_q_head * w.head_dim * w.batch * sum(budgets)), device_status=ctx.status())
 
 
 def prefill_compress_time(w: synth.Workload, reps=3, device="cuda:0"):
@@ -223,6 +232,7 @@ def main():
     ap.add_argument("--steps", type=int, default=12)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
+    ap.add_argument("--per-sequence", action="store_true", help="per-sequence budgets (a rotated budget vector per sequence)")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
     ap.add_argument("--all-kernels", action="store_true", help="launch every kernel of the library once or a few times")
     ap.add_argument("--layers", type=int, default=0, help="with --all-kernels: number of layers of the shape to keep")
@@ -255,7 +265,8 @@ def main():
     if args.prefill:
         print(json.dumps(prefill_compress_time(build_workload(args), args.steps)), flush=True)
         return
-    print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer)), flush=True)
+    print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer,
+                                      per_sequence=args.per_sequence)), flush=True)
 
 
 if __name__ == "__main__":
