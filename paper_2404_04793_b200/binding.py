@@ -167,7 +167,7 @@ class Context:
     def _flatten(self, values, n):
         """[n] -> [n]; with per-sequence budgets [batch][n] -> the C layout (sequence first)."""
         if self.cfg.per_sequence_budgets:
-            if len(values) != self.batch or any(len(v) != n for v in values):
+            if len(values) != self.batch or any(not hasattr(v, "__len__") or len(v) != n for v in values):
                 raise ValueError("expected one list per sequence")
             return [int(b) for row in values for b in row]
         if len(values) != n:

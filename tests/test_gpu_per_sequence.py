@@ -148,3 +148,35 @@ def test_one_sequence_equals_the_batch_mode():
     assert outs[0][0] == outs[1][0]
     for a, b in zip(outs[0][1:], outs[1][1:]):
         assert torch.equal(a, b)
+
+
+def test_argument_and_order_errors():
+    from paper_2404_04793_b200 import binding as B
+    w = _workload(44, n_layer=3)
+    ctx = H.make_ctx(w, per_sequence_budgets=1)
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    a, b = synth.hidden_pair(w, 0, DEV)
+    half = a.reshape(-1, w.hidden)[: w.batch * w.prompt // 2].contiguous()
+    for l in range(w.n_layer):
+        ctx.layer_importance(l, half, half)
+    with pytest.raises(B.SqError) as e:          # half of the prompt tokens are still missing
+        ctx.allocate_budgets(w.b_init, w.p)
+    assert e.value.code == B.SQ_ERR_STATE
+    for l in range(w.n_layer):
+        ctx.layer_importance(l, half, half)
+    with pytest.raises(B.SqError) as e:          # more rows than batch * prompt_len
+        ctx.layer_importance(0, half, half)
+    assert e.value.code == B.SQ_ERR_INVALID_ARG
+    ctx.allocate_budgets(w.b_init, w.p)
+    budgets, _ = ctx.get_budgets()
+    assert len(budgets) == w.batch and all(sum(r) == w.n_layer * w.b_init for r in budgets)
+    with pytest.raises(ValueError):              # one list per sequence is expected
+        ctx.set_budgets([10, 10, 10])
+    with pytest.raises(B.SqError) as e:          # a sequence whose budgets do not fit the pool
+        ctx.set_budgets([[10 * w.b_init] * w.n_layer] * w.batch)
+    assert e.value.code == B.SQ_ERR_CAPACITY
+    cfg = B.make_config(n_layer=2, n_q_head=2, n_kv_head=2, head_dim=64, hidden=64, max_batch=1, max_prompt=8,
+                        max_new_tokens=1, dtype=torch.float32, policy=synth.SLIDING_WINDOW, per_sequence_budgets=2)
+    with pytest.raises(B.SqError) as e:
+        B.sq_query_sizes(cfg, 4)
+    assert e.value.code == B.SQ_ERR_INVALID_ARG
