@@ -564,7 +564,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
       const double t_max = setup + (double)std::min(cand, max_len) / tile;
       const double spread = (double)work / (double)slots + 0.5 * t_max;
       const double cost = items <= slots ? t_max : std::max(t_max, std::min(spread, (double)waves * t_max));
-      if (forced > 0 ? (pieces <= forced) : (split == 0 || cost < best_cost * 0.97)) {  // more pieces only for a clear gain
+      if (forced > 0 ? (pieces <= forced) : (split == 0 || cost < best_cost * 0.90)) {  // more pieces only for a clear gain
         best_cost = cost;
         split = cand;
       }
