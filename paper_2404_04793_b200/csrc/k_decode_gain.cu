@@ -30,8 +30,6 @@ using namespace tc;
 namespace {
 constexpr int kD = 64;
 constexpr int kTileBytes = kTM * kD * 2;  // 16 KB: one K tile
-constexpr int kTmemCols = 256;            // S^T buffers: 3 x up to 80 or 2 x up to 128 head columns
-constexpr int kGainThreads = 320;         // TMA warp, MMA warp, 2 x 4 token warps
 __host__ __device__ constexpr uint32_t idesc_n(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
@@ -41,8 +39,10 @@ struct Candidate {
 };
 }  // namespace
 
-template <int STAGES>
-__global__ void __launch_bounds__(kGainThreads, 2)
+// SETS: groups of four token warps (tile i goes to set i % SETS); TMEM_COLS: tensor-memory columns of the CTA
+// (256: three buffers of up to 80 head columns or two of up to 128; 128: one buffer); CTAS: CTAs per SM aimed at.
+template <int STAGES, int SETS, int TMEM_COLS, int CTAS>
+__global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
     h2o_gain_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, DecodeArgs a,
                        int n_cols, int n_buf) {
   extern __shared__ unsigned char smem_raw[];
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kGainThreads, 2)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "n"(kTmemCols)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "n"(TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -154,6 +154,8 @@ __global__ void __launch_bounds__(kGainThreads, 2)
   } else {
     // ---------------- thread = one token ----------------
     const int quarter = warp & 3, set = (warp - 2) >> 2;
+    constexpr int kThreads = 64 + 128 * SETS;
+    (void)kThreads;
     const int row = quarter * 32 + lane;
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
     const int n32 = G >> 5, n8 = ((G & 31) + 7) >> 3;
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(kGainThreads, 2)
     unsigned long long best = ~0ull;
     int best_slot = -1;
     bool ok = true;
-    for (int i = set; ok && i < n_tiles; i += 2) {
+    for (int i = set; ok && i < n_tiles; i += SETS) {
       const int use = i / n_buf, j = i - use * n_buf;
       const int slot = t0 + i * kTM + row;
       const bool valid = slot < t1;
@@ -249,7 +251,7 @@ __global__ void __launch_bounds__(kGainThreads, 2)
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(TMEM_COLS) : "memory");
   }
   if (tid != 0) return;
   if (*abort_flag) {
@@ -258,7 +260,7 @@ __global__ void __launch_bounds__(kGainThreads, 2)
   }
   if (!full) return;  // the cache still grows: the next token takes a fresh slot
   Candidate best = s_cand[0];
-  for (int q = 1; q < 8; ++q)
+  for (int q = 1; q < 4 * SETS; ++q)
     if (s_cand[q].rank < best.rank) best = s_cand[q];
   int* victim = reinterpret_cast<int*>(a.pool + ldp->victim_off) + unit;
   if (it.n_split == 1) {
@@ -296,16 +298,16 @@ cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_byt
   CUtensorMap tm_q, tm_k;
   if (!make_tile_map(&tm_q, a.q, (long long)q_rows, kD, n_cols) || !make_tile_map(&tm_k, a.pool, pool_rows, kD, kTM))
     return cudaErrorNotSupported;
-  constexpr int kStages = 4;
+  constexpr int kStages = 4, kSets = 2, kTmemCols = 256;
   constexpr size_t smem = 1024 + (size_t)kTM * 128 + (size_t)kStages * kTileBytes + 18 * 8 + kTM * 4 + 8 * sizeof(Candidate);
-  auto kern = h2o_gain_tc_kernel<kStages>;
+  auto kern = h2o_gain_tc_kernel<kStages, kSets, kTmemCols, 2>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<n_items, kGainThreads, smem, s>>>(tm_q, tm_k, a, n_cols, 3 * n_cols <= kTmemCols ? 3 : 2);
+  kern<<<n_items, 64 + 128 * kSets, smem, s>>>(tm_q, tm_k, a, n_cols, kTmemCols == 128 ? 1 : (3 * n_cols <= kTmemCols ? 3 : 2));
   return cudaGetLastError();
 }
 
