@@ -89,7 +89,7 @@ typedef struct sq_config {
                                       sq_get_budgets and sq_evict are [batch][n_layer] (sequence
                                       first), sq_layer_importance takes the rows sequence by
                                       sequence (prompt_len rows each, all of them before
-                                      sq_allocate_budgets), and decode launches are not split-K */
+                                      sq_allocate_budgets) */
 } sq_config;
 
 /* Bytes of cache pool and workspace a context needs when the per-layer budgets sum to at most

@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(128, GT == 1 ? 7 : 1) decode_attn_kernel(Decod
   __shared__ float sm_m[4][GT], sm_l[4][GT];
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, -1, it)) return;
+  if (!locate(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane % LPR, rg = lane / LPR;
   const LayerDesc* ldp = a.layers + it.layer;
@@ -224,16 +224,11 @@ template <typename T>
 __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
   __shared__ SelScratch sc;
   __shared__ __align__(16) float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
-  int layer = a.layer_begin + blockIdx.x / a.n_unit;
-  int unit = blockIdx.x % a.n_unit;
+  // one CTA per (descriptor of the launch, unit)
+  const int unit = blockIdx.x % a.n_unit;
   ItemLoc it;
-  if (a.uniform) {  // items are (descriptor, unit) pairs in launch order
-    if (!locate(a, blockIdx.x, -1, it)) return;
-    layer = it.layer;
-    unit = it.local;
-  } else if (!locate(a, 0, layer, it)) {
-    return;
-  }
+  if (!locate_desc(a, blockIdx.x / a.n_unit, it)) return;
+  const int layer = it.layer;
   const int tid = threadIdx.x, D = a.head_dim, G = a.group, ns = it.n_split;
   const LayerDesc* ldp = a.layers + layer;
   const int b = ldp->b, cap = ldp->cap;
@@ -394,7 +389,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || !need_combine) return e;
-  const int n_cta = (a.layer_end - a.layer_begin) * a.n_unit;
+  const int n_cta = a.n_layer_total * a.n_unit;
   if (dtype == SQ_F32)
     decode_combine_kernel<float><<<n_cta, kSelThreads, 0, s>>>(a);
   else

@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   Candidate* s_cand = reinterpret_cast<Candidate*>(s_nlse + kTM);          // one per token warp
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, -1, it)) return;
+  if (!locate(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const LayerDesc* ldp = a.layers + it.layer;
   const int b = ldp->b, cap = ldp->cap, G = a.group;

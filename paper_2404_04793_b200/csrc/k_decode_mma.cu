@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(32 * WM * WN) decode_attn_mma_kernel(DecodeArg
   unsigned char* v_s = k_s + STAGES * TILE_BYTES;
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, -1, it)) return;
+  if (!locate(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = warp / WN, wn = warp % WN;
   const int gq = lane >> 2, tq = lane & 3;

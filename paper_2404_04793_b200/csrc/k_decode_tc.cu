@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(192, 2)
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, -1, it)) return;
+  if (!locate(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const LayerDesc* ldp = a.layers + it.layer;
   const int b = ldp->b, cap = ldp->cap, G = a.group;

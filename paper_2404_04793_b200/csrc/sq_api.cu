@@ -524,8 +524,9 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     // as many CTAs as fit the GPU at once; among the piece lengths that are whole tiles, take
     // the one with the smallest estimated time.  What a tile, a set-up (in tiles; fitted to
     // measured step times, it includes writing and merging the partial results) and a wave are
-    // depends on the kernel the shape is served by.  With per-sequence budgets the units of a
-    // layer differ in length and are not split: every descriptor has exactly U items.
+    // depends on the kernel the shape is served by.  The running item counts of a split launch
+    // travel in the kernel parameters, which hold kMaxLayers descriptors: larger launches (many
+    // sequences with per-sequence budgets) are not split; they have units to spare anyway.
     const bool bf16 = cfg.dtype == SQ_BF16;
     int tile, setup, per_sm;
     if (bf16 && cfg.head_dim == 64 && G > 32) {  // tcgen05 kernel: 128-token tiles, 2 CTAs per SM
@@ -545,7 +546,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
       const char* ev = getenv("SQ_SPLIT_PIECES");
       return ev ? atoi(ev) : 0;
     }();
-    for (int pieces = 1; pieces <= (c->per_seq ? 1 : 64); ++pieces) {
+    for (int pieces = 1; pieces <= (d1 - d0 > kMaxLayers ? 1 : 64); ++pieces) {
       int cand = ((max_len + pieces - 1) / pieces + tile - 1) / tile * tile;
       if (pieces > 1 && cand < 2 * tile) break;  // a piece is never shorter than two tiles
       if (cand == prev) continue;
@@ -569,14 +570,21 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
         split = cand;
       }
     }
+    // the launch's descriptors in launch order: the global order for the whole stack, else layer by layer
+    const bool all = (s == 0 && e == cfg.n_layer);
+    const int* order_host = all ? c->hs.order : c->hs.order_by_layer + d0;
+    DecodeArgs a;
     long long n_items = 0;
-    for (int d = d0; d < d1; ++d) {
-      int len = std::min(n_tok + 1, c->hs.layers[d].b);
-      int ns = (len + split - 1) / split;
+    bool any_split = false;
+    for (int k = 0; k < d1 - d0; ++k) {
+      const int len = std::min(n_tok + 1, c->hs.layers[order_host[k]].b);
+      const int ns = (len + split - 1) / split;
+      any_split |= ns > 1;
+      if (k <= kMaxLayers) a.cum[std::min(k, kMaxLayers)] = (int)n_items;
       n_items += (long long)U * ns;
     }
+    if (d1 - d0 <= kMaxLayers) a.cum[d1 - d0] = (int)n_items;
     if ((size_t)n_items > c->wl.items_cap) return fail(c, SQ_ERR_CAPACITY, "workspace too small for the split plan");
-    DecodeArgs a;
     a.layers = ws_ptr<LayerDesc>(c, c->wl.layers);
     a.pool = c->pool;
     a.logits = ws_ptr<float>(c, c->wl.logits);
@@ -589,16 +597,9 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.status = ws_ptr<int>(c, c->wl.status);
     a.tickets = ws_ptr<int>(c, c->wl.tickets);
     // without split-K every descriptor has exactly U items and an item is found in O(1)
-    a.uniform = (n_items == (long long)U * (d1 - d0)) ? 1 : 0;
-    if (a.uniform) {
-      // the launch's descriptors only: the global order for the whole stack, else layer by layer
-      const bool all = (s == 0 && e == cfg.n_layer);
-      a.order = all ? ws_ptr<int>(c, c->wl.order) : ws_ptr<int>(c, c->wl.order_by_layer) + d0;
-      a.n_layer_total = d1 - d0;
-    } else {
-      a.order = ws_ptr<int>(c, c->wl.order);
-      a.n_layer_total = c->n_desc;
-    }
+    a.uniform = any_split ? 0 : 1;
+    a.order = all ? ws_ptr<int>(c, c->wl.order) : ws_ptr<int>(c, c->wl.order_by_layer) + d0;
+    a.n_layer_total = d1 - d0;
     a.layer_begin = d0;
     a.layer_end = d1;
     a.n_tok = n_tok;

@@ -14,59 +14,41 @@ struct ItemLoc {
   int layer, local, n_split, base;
 };
 
-__device__ __forceinline__ int n_split_of(const DecodeArgs& a, int b) {
-  int len = min(a.n_tok + 1, b);
-  return (len + a.split_tokens - 1) / a.split_tokens;
-}
-
-// Work items of a launch are numbered layer by layer in `order` (largest budget first), and
-// within a layer as unit * n_split + split.  Each warp finds, by a prefix scan over the
-// layers, either the layer an item index falls in (want_layer < 0) or the first item of a
-// given layer.
-__device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, int want_layer, ItemLoc& out) {
-  if (a.uniform) {  // `order` lists exactly the launch's descriptors, n_unit items each
-    const int k = idx / a.n_unit;
-    if (k >= a.n_layer_total) return false;
-    out.layer = a.order[k];
+// Work items of a launch are numbered descriptor by descriptor in the order of a.order (largest
+// budget first), and within a descriptor as unit * n_split + split.  Without split-K every
+// descriptor has n_unit items and the lookup is a division; with it the running item counts
+// a.cum (kernel parameters: constant memory) are searched.
+__device__ __forceinline__ bool locate_desc(const DecodeArgs& a, int k, ItemLoc& out) {
+  if (k >= a.n_layer_total) return false;
+  out.layer = a.order[k];
+  if (a.uniform) {
     out.n_split = 1;
     out.base = k * a.n_unit;
-    out.local = idx - out.base;
-    return true;
+  } else {
+    out.base = a.cum[k];
+    out.n_split = (a.cum[k + 1] - out.base) / a.n_unit;
   }
-  const int lane = threadIdx.x & 31;
-  int running = 0;
-  for (int c = 0; c < a.n_layer_total; c += 32) {
-    const int i = c + lane;
-    int l = -1, ns = 0, cnt = 0;
-    if (i < a.n_layer_total) {
-      int li = a.order[i];
-      if (li >= a.layer_begin && li < a.layer_end) {
-        l = li;
-        ns = n_split_of(a, a.layers[li].b);
-        cnt = a.n_unit * ns;
-      }
-    }
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int t = __shfl_up_sync(kFull, incl, o);
-      if (lane >= o) incl += t;
-    }
-    unsigned hit = (want_layer >= 0) ? __ballot_sync(kFull, l == want_layer)
-                                     : __ballot_sync(kFull, cnt > 0 && idx < running + incl);
-    if (hit) {
-      const int src = __ffs(hit) - 1;
-      out.layer = __shfl_sync(kFull, l, src);
-      out.n_split = __shfl_sync(kFull, ns, src);
-      out.base = running + __shfl_sync(kFull, incl - cnt, src);
-      out.local = idx - out.base;
-      return true;
-    }
-    running += __shfl_sync(kFull, incl, 31);
-  }
-  return false;
+  out.local = 0;
+  return true;
 }
-
+__device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, ItemLoc& out) {
+  int k;
+  if (a.uniform) {
+    k = idx / a.n_unit;
+  } else {
+    if (idx >= a.cum[a.n_layer_total]) return false;
+    int lo = 0, hi = a.n_layer_total;  // cum[lo] <= idx < cum[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (a.cum[mid] <= idx) lo = mid;
+      else hi = mid;
+    }
+    k = lo;
+  }
+  if (!locate_desc(a, k, out)) return false;
+  out.local = idx - out.base;
+  return true;
+}
 
 // Split-K merge without a second launch (policies without scores): every piece of a unit
 // bumps the unit's ticket after its partials are written; the piece that arrives last reads

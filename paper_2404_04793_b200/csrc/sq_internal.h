@@ -72,7 +72,7 @@ struct ScoreArgs {  // H2O prompt scores of one layer
 // budgets, a (layer, sequence) pair holding that sequence's n_kv_head units (batch = 1 then).
 struct DecodeArgs {
   const LayerDesc* layers;
-  const int* order;  // descriptor indices sorted by budget, descending; with `uniform` only those of the launch
+  const int* order;  // the launch's descriptors, n_layer_total of them, in launch order (largest budget first)
   char* pool;
   float* logits;
   float* part_stat;  // [item][group][4]   (max, sum, sum of rounded weights, pad) in the log2 domain
@@ -89,6 +89,9 @@ struct DecodeArgs {
   int n_unit;  // batch * n_kv_head
   int split_tokens, policy;
   int uniform;  // every descriptor of the launch has n_unit items (no split-K): items are found in O(1)
+  // else: items before the k-th descriptor of the launch (k <= n_layer_total <= kMaxLayers); rides
+  // in the kernel parameters, so a lookup is a binary search in constant memory
+  int cum[kMaxLayers + 1];
   float scale_log2;  // log2(e) / sqrt(head_dim)
 };
 

@@ -180,3 +180,37 @@ def test_argument_and_order_errors():
     with pytest.raises(B.SqError) as e:
         B.sq_query_sizes(cfg, 4)
     assert e.value.code == B.SQ_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("policy", [synth.SLIDING_WINDOW, synth.H2O])
+@pytest.mark.parametrize("hq,hkv,head_dim", [(8, 2, 128), (71, 1, 64), (2, 2, 128)])
+def test_long_contexts_split_across_ctas(policy, hq, hkv, head_dim):
+    """Few units with long, unequal budgets: the launch splits each unit's tokens over several
+    CTAs, a different number of pieces per sequence."""
+    w = _workload(45, policy=policy, dtype=torch.bfloat16, head_dim=head_dim, n_q_head=hq, n_kv_head=hkv, batch=2,
+                  n_layer=2, prompt=3000, steps=3, hidden=64, heavy_mode="zipf")
+    budgets = [[2500, 300], [700, 2900]]
+    ctx = H.make_ctx(w, b_init=2900, per_sequence_budgets=1)
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets(budgets)
+    prompt_cpu = H.prefill_all(ctx, w, DEV)
+    units = H.all_units(w)
+    oracles = {(l, s, h): H.oracle_unit(w, budgets[s], prompt_cpu, l, s, h) for (l, s, h) in units}
+    g = w.group
+    for t in range(w.steps):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        if t == 1:   # one step layer by layer
+            for l in range(w.n_layer):
+                ctx.decode_step(l, l + 1, q[l], kn[l], vn[l], out[l])
+        else:
+            ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+        qc, kc, vc, oc = q.cpu(), kn.cpu(), vn.cpu(), out.cpu()
+        for (l, s, h) in units:
+            u = oracles[(l, s, h)]
+            want = u.decode_step(H.f64(qc[l, s, h * g:(h + 1) * g]), H.f64(kc[l, s, h]), H.f64(vc[l, s, h]))
+            assert np.max(np.abs(H.f64(oc[l, s, h * g:(h + 1) * g]) - want)) <= H.TOL_OUT[w.dtype], (t, l, s, h)
+    for (l, s, h) in units:
+        if policy != synth.H2O:
+            assert ctx.get_kept(l, s, h)[0] == oracles[(l, s, h)].kept_positions(), (l, s, h)
+    assert ctx.status() == 0
