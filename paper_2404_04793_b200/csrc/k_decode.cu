@@ -17,8 +17,9 @@ namespace sq {
 // Each lane keeps its 16-byte slice of up to GT query heads (pre-scaled by log2(e)/sqrt(d))
 // and of their output accumulators in fp32; logits are reduced over the LPR lanes by
 // shuffles, and the softmax runs online in the log2 domain over batches of U rows.
-template <typename T, int D, int GT>
-__global__ void __launch_bounds__(128, GT == 1 ? 7 : 1) decode_attn_kernel(DecodeArgs a) {
+// UNIFORM: the launch has no split-K (see locate()).
+template <typename T, int D, int GT, int UNIFORM, class Args>
+__global__ void __launch_bounds__(128, GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) decode_attn_kernel(Args a) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;   // lanes per row
   constexpr int RPW = 32 / LPR;  // rows per warp per load
@@ -27,7 +28,7 @@ __global__ void __launch_bounds__(128, GT == 1 ? 7 : 1) decode_attn_kernel(Decod
   __shared__ float sm_m[4][GT], sm_l[4][GT];
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, it)) return;
+  if (!locate<UNIFORM, Args>(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane % LPR, rg = lane / LPR;
   const LayerDesc* ldp = a.layers + it.layer;
@@ -338,12 +339,15 @@ __global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs 
 
 template <typename T, int D>
 static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
-  if (a.group == 1)
-    decode_attn_kernel<T, D, 1><<<n_items, 128, 0, s>>>(a);
-  else if (a.group <= 4)
-    decode_attn_kernel<T, D, 4><<<n_items, 128, 0, s>>>(a);
-  else
-    decode_attn_kernel<T, D, 8><<<n_items, 128, 0, s>>>(a);
+  if (a.group == 1) {
+    // the register-capped kernel gets its own build for launches without split-K
+    if (a.uniform) decode_attn_kernel<T, D, 1, 1, DecodeArgsBase><<<n_items, 128, 0, s>>>(a);  // sliced: no table
+    else decode_attn_kernel<T, D, 1, 0, DecodeArgs><<<n_items, 128, 0, s>>>(a);
+  } else if (a.group <= 4) {
+    decode_attn_kernel<T, D, 4, -1, DecodeArgs><<<n_items, 128, 0, s>>>(a);
+  } else {
+    decode_attn_kernel<T, D, 8, -1, DecodeArgs><<<n_items, 128, 0, s>>>(a);
+  }
 }
 
 // Which attention kernel serves a shape: grouped bf16 heads go to the tensor-core kernel,

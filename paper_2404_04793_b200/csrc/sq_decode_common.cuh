@@ -18,34 +18,47 @@ struct ItemLoc {
 // budget first), and within a descriptor as unit * n_split + split.  Without split-K every
 // descriptor has n_unit items and the lookup is a division; with it the running item counts
 // a.cum (kernel parameters: constant memory) are searched.
-__device__ __forceinline__ bool locate_desc(const DecodeArgs& a, int k, ItemLoc& out) {
+// UNIFORM: 1 = the launch is known to have no split-K (the search code is not even compiled in:
+// the register-capped kernel keeps its budget), 0 = it is known to have it, -1 = read a.uniform.
+template <int UNIFORM = -1, class Args = DecodeArgs>
+__device__ __forceinline__ bool locate_desc(const Args& a, int k, ItemLoc& out) {
   if (k >= a.n_layer_total) return false;
   out.layer = a.order[k];
-  if (a.uniform) {
+  if constexpr (UNIFORM == 1) {
     out.n_split = 1;
     out.base = k * a.n_unit;
   } else {
-    out.base = a.cum[k];
-    out.n_split = (a.cum[k + 1] - out.base) / a.n_unit;
+    if (UNIFORM < 0 && a.uniform) {
+      out.n_split = 1;
+      out.base = k * a.n_unit;
+    } else {
+      out.base = a.cum[k];
+      out.n_split = (a.cum[k + 1] - out.base) / a.n_unit;
+    }
   }
   out.local = 0;
   return true;
 }
-__device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, ItemLoc& out) {
+template <int UNIFORM = -1, class Args = DecodeArgs>
+__device__ __forceinline__ bool locate(const Args& a, int idx, ItemLoc& out) {
   int k;
-  if (a.uniform) {
+  if constexpr (UNIFORM == 1) {
     k = idx / a.n_unit;
   } else {
-    if (idx >= a.cum[a.n_layer_total]) return false;
-    int lo = 0, hi = a.n_layer_total;  // cum[lo] <= idx < cum[hi]
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (a.cum[mid] <= idx) lo = mid;
-      else hi = mid;
+    if (UNIFORM < 0 && a.uniform) {
+      k = idx / a.n_unit;
+    } else {
+      if (idx >= a.cum[a.n_layer_total]) return false;
+      int lo = 0, hi = a.n_layer_total;  // cum[lo] <= idx < cum[hi]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (a.cum[mid] <= idx) lo = mid;
+        else hi = mid;
+      }
+      k = lo;
     }
-    k = lo;
   }
-  if (!locate_desc(a, k, out)) return false;
+  if (!locate_desc<UNIFORM, Args>(a, k, out)) return false;
   out.local = idx - out.base;
   return true;
 }
@@ -58,7 +71,7 @@ __device__ __forceinline__ bool locate(const DecodeArgs& a, int idx, ItemLoc& ou
 // The merge is run by a group of nt threads (tid = index within the group) that synchronise
 // through sync(), which returns false when the group gives up.
 template <typename T, int kBatch, typename Sync>
-__device__ __forceinline__ void merge_if_last_group(const DecodeArgs& a, const ItemLoc& it, int unit, float* lse_out,
+__device__ __forceinline__ void merge_if_last_group(const DecodeArgsBase& a, const ItemLoc& it, int unit, float* lse_out,
                                                     int tid, int nt, Sync sync) {
   __shared__ int s_last;
   __shared__ float s_mM[kMaxGroup], s_mInv[kMaxGroup];
@@ -153,7 +166,7 @@ __device__ __forceinline__ void merge_if_last_group(const DecodeArgs& a, const I
 
 // The whole CTA merges.
 template <typename T, int kBatch = 4>
-__device__ __forceinline__ void merge_if_last(const DecodeArgs& a, const ItemLoc& it, int unit,
+__device__ __forceinline__ void merge_if_last(const DecodeArgsBase& a, const ItemLoc& it, int unit,
                                               float* lse_out = nullptr) {
   merge_if_last_group<T, kBatch>(a, it, unit, lse_out, (int)threadIdx.x, (int)blockDim.x, [] {
     __syncthreads();

@@ -70,7 +70,7 @@ struct ScoreArgs {  // H2O prompt scores of one layer
 
 // "Layer" below means one cache descriptor: a layer of the whole batch, or, with per-sequence
 // budgets, a (layer, sequence) pair holding that sequence's n_kv_head units (batch = 1 then).
-struct DecodeArgs {
+struct DecodeArgsBase {
   const LayerDesc* layers;
   const int* order;  // the launch's descriptors, n_layer_total of them, in launch order (largest budget first)
   char* pool;
@@ -89,10 +89,13 @@ struct DecodeArgs {
   int n_unit;  // batch * n_kv_head
   int split_tokens, policy;
   int uniform;  // every descriptor of the launch has n_unit items (no split-K): items are found in O(1)
-  // else: items before the k-th descriptor of the launch (k <= n_layer_total <= kMaxLayers); rides
-  // in the kernel parameters, so a lookup is a binary search in constant memory
-  int cum[kMaxLayers + 1];
   float scale_log2;  // log2(e) / sqrt(head_dim)
+};
+// With split-K: items before the k-th descriptor of the launch (k <= n_layer_total <= kMaxLayers).
+// Rides in the kernel parameters, so a lookup is a binary search in constant memory; the kernel
+// build for launches without split-K takes the base only (1 KB less to pass per launch).
+struct DecodeArgs : DecodeArgsBase {
+  int cum[kMaxLayers + 1];
 };
 
 struct EvictLayer {  // one layer of an explicit eviction
