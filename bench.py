@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read+write) per decode launch of the default workload, from the ncu capture
 # summarised in profiles/decode_attn_llama2_7b_sw_b2.md (batch-2 capture scaled by 4 to batch 8).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama2_7b_sw_bf16": 1.7359e9}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama2_7b_sw_bf16": 1.7373e9}
 
 
 def workload_by_name(name):
