@@ -188,10 +188,13 @@ cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, int* status, cu
 // Writes the kept positions in ascending order to the layer's position table.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelThreads) select_prompt_kernel(const float* __restrict__ acc_prompt, int P,
-                                                                    LayerDesc ld, char* pool) {
+                                                                    const LayerDesc* __restrict__ descs,
+                                                                    int units_per_desc, char* pool) {
   __shared__ SelScratch sc;
-  const int unit = blockIdx.x, tid = threadIdx.x;
-  const float* acc = acc_prompt + (size_t)unit * P;
+  const int tid = threadIdx.x;
+  const LayerDesc ld = descs[blockIdx.x / units_per_desc];  // the descriptor this unit belongs to
+  const int unit = blockIdx.x % units_per_desc;             // its index within the descriptor
+  const float* acc = acc_prompt + (size_t)blockIdx.x * P;
   int* pos_out = reinterpret_cast<int*>(pool + ld.pos_off) + (size_t)unit * ld.cap;
   if (P <= ld.b) {
     for (int i = tid; i < P; i += kSelThreads) pos_out[i] = i;
@@ -235,16 +238,20 @@ __global__ void __launch_bounds__(kSelThreads) select_prompt_kernel(const float*
   }
 }
 
-cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc& ld, char* pool,
-                                 cudaStream_t s) {
-  select_prompt_kernel<<<n_unit, kSelThreads, 0, s>>>(acc_prompt, prompt, ld, pool);
+cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc* descs,
+                                 int units_per_desc, char* pool, cudaStream_t s) {
+  select_prompt_kernel<<<n_unit, kSelThreads, 0, s>>>(acc_prompt, prompt, descs, units_per_desc, pool);
   return cudaGetLastError();
 }
 
 // First victim of a full H2O cache (the token the next append will replace).
-__global__ void __launch_bounds__(kSelThreads) pick_victim_kernel(char* pool, LayerDesc ld, int len, int next_pos) {
+__global__ void __launch_bounds__(kSelThreads) pick_victim_kernel(char* pool, const LayerDesc* __restrict__ descs,
+                                                                  int units_per_desc, int prompt, int next_pos) {
   __shared__ SelScratch sc;
-  const int unit = blockIdx.x;
+  const LayerDesc ld = descs[blockIdx.x / units_per_desc];
+  const int unit = blockIdx.x % units_per_desc;
+  const int len = min(prompt, ld.b);
+  if (len < ld.b) return;  // the cache still grows: the next token takes a fresh slot
   const int* pos = reinterpret_cast<const int*>(pool + ld.pos_off) + (size_t)unit * ld.cap;
   const float* acc = reinterpret_cast<const float*>(pool + ld.acc_off) + (size_t)unit * ld.cap;
   const int thr = next_pos - ld.b_recent;
@@ -264,8 +271,9 @@ __global__ void __launch_bounds__(kSelThreads) pick_victim_kernel(char* pool, La
   if (threadIdx.x == 0) reinterpret_cast<int*>(pool + ld.victim_off)[unit] = slot;
 }
 
-cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int len, int next_pos, cudaStream_t s) {
-  pick_victim_kernel<<<n_unit, kSelThreads, 0, s>>>(pool, ld, len, next_pos);
+cudaError_t launch_pick_victim(char* pool, const LayerDesc* descs, int units_per_desc, int n_unit, int prompt,
+                               int next_pos, cudaStream_t s) {
+  pick_victim_kernel<<<n_unit, kSelThreads, 0, s>>>(pool, descs, units_per_desc, prompt, next_pos);
   return cudaGetLastError();
 }
 
@@ -277,30 +285,34 @@ cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int 
 constexpr int kGatherSlots = 16;
 
 __global__ void __launch_bounds__(256) gather_kernel(GatherArgs a, int row_bytes) {
-  const int unit = blockIdx.x, s0 = blockIdx.y * kGatherSlots;
+  const int ug = blockIdx.x, s0 = blockIdx.y * kGatherSlots;  // ug: unit of the batch (sequence, KV head)
+  const LayerDesc ld = a.descs[ug / a.units_per_desc];
+  const int unit = ug % a.units_per_desc;                     // its index within the descriptor
+  const int n_keep = min(a.prompt, ld.b);
+  if (s0 >= n_keep) return;                                   // the grid covers the longest descriptor
   const int vpr = row_bytes / 16;  // 16-byte vectors per row
-  int* pos_tab = reinterpret_cast<int*>(a.pool + a.ld.pos_off) + (size_t)unit * a.ld.cap;
-  float* acc_tab = reinterpret_cast<float*>(a.pool + a.ld.acc_off) + (size_t)unit * a.ld.cap;
+  int* pos_tab = reinterpret_cast<int*>(a.pool + ld.pos_off) + (size_t)unit * ld.cap;
+  float* acc_tab = reinterpret_cast<float*>(a.pool + ld.acc_off) + (size_t)unit * ld.cap;
   __shared__ int s_pos[kGatherSlots];
   if (threadIdx.x < kGatherSlots) {
     const int slot = s0 + threadIdx.x;
     int p = -1;
-    if (slot < a.n_keep) {
+    if (slot < n_keep) {
       if (a.policy == SQ_POLICY_H2O) {
         p = pos_tab[slot];
-        acc_tab[slot] = a.acc_prompt ? a.acc_prompt[(size_t)unit * a.prompt + p] : 0.f;
+        acc_tab[slot] = a.acc_prompt ? a.acc_prompt[(size_t)ug * a.prompt + p] : 0.f;
       } else {
-        p = (slot < a.ld.ring_base) ? slot : a.ld.ring_origin + (slot - a.ld.ring_base);
+        p = (slot < ld.ring_base) ? slot : ld.ring_origin + (slot - ld.ring_base);
         pos_tab[slot] = p;
       }
     }
     s_pos[threadIdx.x] = p;
   }
   __syncthreads();
-  const uint4* ksrc = reinterpret_cast<const uint4*>(a.k_prompt) + (size_t)unit * a.prompt * vpr;
-  const uint4* vsrc = reinterpret_cast<const uint4*>(a.v_prompt) + (size_t)unit * a.prompt * vpr;
-  uint4* kdst = reinterpret_cast<uint4*>(a.pool + a.ld.k_off) + (size_t)unit * a.ld.cap * vpr;
-  uint4* vdst = reinterpret_cast<uint4*>(a.pool + a.ld.v_off) + (size_t)unit * a.ld.cap * vpr;
+  const uint4* ksrc = reinterpret_cast<const uint4*>(a.k_prompt) + (size_t)ug * a.prompt * vpr;
+  const uint4* vsrc = reinterpret_cast<const uint4*>(a.v_prompt) + (size_t)ug * a.prompt * vpr;
+  uint4* kdst = reinterpret_cast<uint4*>(a.pool + ld.k_off) + (size_t)unit * ld.cap * vpr;
+  uint4* vdst = reinterpret_cast<uint4*>(a.pool + ld.v_off) + (size_t)unit * ld.cap * vpr;
   for (int idx = threadIdx.x; idx < kGatherSlots * vpr; idx += 256) {
     const int j = idx / vpr, v = idx % vpr;
     const int p = s_pos[j];
@@ -312,9 +324,9 @@ __global__ void __launch_bounds__(256) gather_kernel(GatherArgs a, int row_bytes
 }
 
 cudaError_t launch_gather(const GatherArgs& a, int dtype, cudaStream_t s) {
-  if (a.n_keep <= 0) return cudaSuccess;
+  if (a.max_keep <= 0) return cudaSuccess;
   const int row_bytes = a.head_dim * (dtype == SQ_F32 ? 4 : 2);
-  dim3 grid(a.n_unit, (a.n_keep + kGatherSlots - 1) / kGatherSlots);
+  dim3 grid(a.n_unit, (a.max_keep + kGatherSlots - 1) / kGatherSlots);
   gather_kernel<<<grid, 256, 0, s>>>(a, row_bytes);
   return cudaGetLastError();
 }

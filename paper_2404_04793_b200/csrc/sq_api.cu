@@ -468,27 +468,31 @@ int sq_prefill_compress(sq_ctx* c, int32_t layer, const void* k_prompt, const vo
       acc = s.acc_prompt;
     }
   }
-  // selection and gather per descriptor (the whole batch, or one sequence at a time)
-  const size_t kv_stride = (size_t)U * P * c->cfg.head_dim * elem_bytes(c->cfg.dtype);
+  // selection, gather and first victim: one launch each over all descriptors of the layer
+  const LayerDesc* descs_dev = ws_ptr<LayerDesc>(c, c->wl.layers) + layer * c->n_grp;
+  const int n_unit = c->batch * c->cfg.n_kv_head;
+  int max_keep = 0;
+  bool any_full = false;
   for (int g = 0; g < c->n_grp; ++g) {
     const LayerDesc& ld = c->hs.layers[layer * c->n_grp + g];
-    const int n_keep = std::min(P, ld.b);
-    const float* acc_g = acc ? acc + (size_t)g * U * P : nullptr;
-    if (h2o) SQ_CUDA(c, launch_select_prompt(acc_g, U, P, ld, c->pool, st));
-    GatherArgs ga;
-    ga.k_prompt = static_cast<const char*>(k_prompt) + g * kv_stride;
-    ga.v_prompt = static_cast<const char*>(v_prompt) + g * kv_stride;
-    ga.acc_prompt = acc_g;
-    ga.pool = c->pool;
-    ga.ld = ld;
-    ga.n_unit = U;
-    ga.prompt = P;
-    ga.n_keep = n_keep;
-    ga.policy = c->cfg.policy;
-    ga.head_dim = c->cfg.head_dim;
-    SQ_CUDA(c, launch_gather(ga, c->cfg.dtype, st));
-    if (h2o && n_keep == ld.b) SQ_CUDA(c, launch_pick_victim(c->pool, ld, U, n_keep, P, st));
+    max_keep = std::max(max_keep, std::min(P, ld.b));
+    any_full |= P >= ld.b;
   }
+  if (h2o) SQ_CUDA(c, launch_select_prompt(acc, n_unit, P, descs_dev, U, c->pool, st));
+  GatherArgs ga;
+  ga.k_prompt = k_prompt;
+  ga.v_prompt = v_prompt;
+  ga.acc_prompt = acc;
+  ga.pool = c->pool;
+  ga.descs = descs_dev;
+  ga.units_per_desc = U;
+  ga.n_unit = n_unit;
+  ga.prompt = P;
+  ga.max_keep = max_keep;
+  ga.policy = c->cfg.policy;
+  ga.head_dim = c->cfg.head_dim;
+  SQ_CUDA(c, launch_gather(ga, c->cfg.dtype, st));
+  if (h2o && any_full) SQ_CUDA(c, launch_pick_victim(c->pool, descs_dev, U, n_unit, P, P, st));
   c->n_tok[layer] = P;
   c->prefilled[layer] = true;
   return SQ_OK;

@@ -51,13 +51,14 @@ struct AllocateArgs {  // entry of layer i: [i * stride + blockIdx.x] (one CTA p
   unsigned char* is_g3;
 };
 
-struct GatherArgs {  // prompt rows -> cache slots of one layer
+struct GatherArgs {  // prompt rows -> cache slots of one layer (all its descriptors in one launch)
   const void* k_prompt;
   const void* v_prompt;
   const float* acc_prompt;  // H2O, else null
   char* pool;
-  LayerDesc ld;
-  int n_unit, prompt, n_keep, policy, head_dim;
+  const LayerDesc* descs;   // the layer's descriptors (device); unit u belongs to descs[u / units_per_desc]
+  int units_per_desc;
+  int n_unit, prompt, max_keep, policy, head_dim;
 };
 
 struct ScoreArgs {  // H2O prompt scores of one layer
@@ -118,9 +119,10 @@ cudaError_t launch_gather(const GatherArgs& a, int dtype, cudaStream_t s);
 cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, int* status, cudaStream_t s);
 cudaError_t launch_prefill_scores_alu(const ScoreArgs& a, int dtype, cudaStream_t s);
 cudaError_t launch_prefill_scores_tc(const ScoreArgs& a, int* status, cudaStream_t s);
-cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc& ld, char* pool,
-                                 cudaStream_t s);
-cudaError_t launch_pick_victim(char* pool, const LayerDesc& ld, int n_unit, int len, int next_pos, cudaStream_t s);
+cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt, const LayerDesc* descs,
+                                 int units_per_desc, char* pool, cudaStream_t s);
+cudaError_t launch_pick_victim(char* pool, const LayerDesc* descs, int units_per_desc, int n_unit, int prompt,
+                               int next_pos, cudaStream_t s);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
                           size_t q_rows, cudaStream_t s);
 cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
