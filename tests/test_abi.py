@@ -32,6 +32,23 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(B.EXPORTS) == names
 
 
+def test_config_struct_matches_the_header():
+    """The ctypes mirror of sq_config lists the header's int32 fields in the header's order."""
+    text = open(os.path.join(ROOT, "include", "sq.h")).read()
+    body = text[text.index("typedef struct sq_config {"):text.index("} sq_config;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = re.findall(r"int32_t\s+([a-z_]+)\s*;", body)
+    assert fields == [n for n, _ in B.sq_config._fields_]
+    assert ctypes.sizeof(B.sq_config) == 4 * len(fields)
+
+
+def test_per_sequence_budgets_size_the_tables(lib):
+    """One descriptor per (layer, sequence): the workspace grows with the batch, the K/V part of the pool does not."""
+    p0, w0 = B.sq_query_sizes(_cfg(max_batch=8), 100)
+    p1, w1 = B.sq_query_sizes(_cfg(max_batch=8, per_sequence_budgets=1), 100)
+    assert w1 > w0 and p1 >= p0 and p1 - p0 < 4 * 8 * 6 * 256 + 1
+
+
 def _cfg(**kw):
     base = dict(n_layer=4, n_q_head=2, n_kv_head=2, head_dim=64, hidden=128, max_batch=1, max_prompt=256,
                 max_new_tokens=16, dtype=B.SQ_F32, policy=B.SQ_POLICY_H2O)
@@ -60,6 +77,7 @@ def test_query_sizes_scale_with_budget(lib):
     (dict(heavy_num=2, heavy_den=2), B.SQ_ERR_INVALID_ARG),
     (dict(page_tokens=0), B.SQ_ERR_INVALID_ARG),
     (dict(dtype=7), B.SQ_ERR_INVALID_ARG),
+    (dict(per_sequence_budgets=2), B.SQ_ERR_INVALID_ARG),
 ])
 def test_bad_configs_are_rejected(lib, kw, code):
     with pytest.raises(B.SqError) as e:
