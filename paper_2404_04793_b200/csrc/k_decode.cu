@@ -353,7 +353,7 @@ static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
 // Which attention kernel serves a shape: grouped bf16 heads go to the tensor-core kernel,
 // everything else (fp32, one query head per KV head, shapes it does not cover) to the fp32-pipe
 // kernel.  SQ_DECODE_PATH=alu|mma overrides the choice (mma also keeps wide groups off the tcgen05 kernel) (for A/B measurements).
-static int decode_path_override() {
+int decode_path_override() {
   static int mode = -1;
   if (mode < 0) {
     const char* e = getenv("SQ_DECODE_PATH");
@@ -378,6 +378,9 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
       return e;
     }
   }
+  // every other kernel needs the per-slot logits for H2O: a context sized for the tcgen05 pair
+  // does not hold them, and nothing may fall back silently
+  if (!done && a.policy == SQ_POLICY_H2O && !a.has_logits) return cudaErrorNotSupported;
   if (!done && dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
     cudaError_t e = launch_decode_attn_mma(a, n_items, s);
     if (e == cudaSuccess) done = true;

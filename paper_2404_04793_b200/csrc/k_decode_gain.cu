@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
   const int* pos = reinterpret_cast<const int*>(a.pool + ldp->pos_off) + (size_t)unit * cap;
   float* acc = reinterpret_cast<float*>(a.pool + ldp->acc_off) + (size_t)unit * cap;
-  const float* lse = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  const float* lse = a.logits + ldp->lse_off + (size_t)unit * G;
   const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
   const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
 

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(192, 2)
   const bf16* vn = reinterpret_cast<const bf16*>(a.v_new) + (tok * a.n_kv_head + kvh) * kD;
   bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
   // H2O: the unit's row log-sum-exps (log2 domain), read by the score-update pass that follows
-  float* lse = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  float* lse = a.logits + ldp->lse_off + (size_t)unit * G;
   float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
   float* po = a.part_o + (size_t)blockIdx.x * G * kD;
   // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q

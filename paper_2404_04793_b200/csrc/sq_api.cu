@@ -24,7 +24,7 @@ struct WsLayout {
   size_t cos_sum, tok_count, cta_partial, ticket, cos_sim, budget, is_g3, status, tickets, layers, order, order_by_layer,
       evict_tab;
   size_t part_stat, part_o, logits, acc_prompt, lse2, total;
-  size_t items_cap, logits_floats, n_desc_cap;
+  size_t items_cap, logits_floats, lse_floats, n_desc_cap;
 };
 
 // Pinned staging for the small host <-> device tables.  "desc" = one cache descriptor: a layer
@@ -102,6 +102,14 @@ int check_config(const sq_config* c, std::string* why) {
   return SQ_OK;
 }
 
+// H2O decode of 33..128 bf16 query heads per KV head at head_dim 64 runs on the tcgen05 attention
+// + score-pass pair, which keeps no per-slot logits (SQ_DECODE_PATH forces the other kernels).
+bool wide_h2o_pair(const sq_config& c) {
+  const int G = c.n_q_head / c.n_kv_head;
+  return c.policy == SQ_POLICY_H2O && c.dtype == SQ_BF16 && c.head_dim == 64 && G > 32 && G <= kMaxGroup &&
+         decode_path_override() == 0;
+}
+
 size_t pool_bytes_for(const sq_config& c, int64_t b_init) {
   const size_t U = (size_t)c.max_batch * c.n_kv_head;
   const size_t tokens = (size_t)c.n_layer * (size_t)b_init + (size_t)c.n_layer * (c.page_tokens - 1);
@@ -138,8 +146,11 @@ WsLayout ws_layout(const sq_config& c, int64_t b_init) {
   w.part_stat = take(w.items_cap * G * 4 * 4);
   w.part_o = take(w.items_cap * G * c.head_dim * 4);
   const bool h2o = c.policy == SQ_POLICY_H2O;
-  w.logits_floats = h2o ? U * G * (L * (size_t)b_init + L * (c.page_tokens - 1)) : 0;
-  w.logits = take(w.logits_floats * 4);
+  // H2O: row log-sum-exps [unit][group] per layer, then (unless the shape is served by the
+  // tcgen05 pair, which recomputes the logits) the logits of every slot
+  w.lse_floats = h2o ? U * G * L : 0;
+  w.logits_floats = (h2o && !wide_h2o_pair(c)) ? U * G * (L * (size_t)b_init + L * (c.page_tokens - 1)) : 0;
+  w.logits = take((w.lse_floats + w.logits_floats) * 4);
   w.acc_prompt = take(h2o ? U * (size_t)c.max_prompt * 4 : 0);
   w.lse2 = take(h2o ? (size_t)c.max_batch * c.n_q_head * c.max_prompt * 4 : 0);
   w.total = off;
@@ -178,7 +189,8 @@ int build_layout(sq_ctx* c, cudaStream_t st) {
   const size_t U = (size_t)c->desc_units, G = cfg.n_q_head / cfg.n_kv_head;
   const size_t row = (size_t)cfg.head_dim * elem_bytes(cfg.dtype);
   const bool h2o = cfg.policy == SQ_POLICY_H2O;
-  size_t off = 0, lfl = 0;
+  size_t off = 0, lfl = 0, lse = 0;
+  const bool slot_logits = h2o && !wide_h2o_pair(cfg);
   for (int d = 0; d < c->n_desc; ++d) {
     LayerDesc& ld = c->hs.layers[d];
     const int b = c->hs.budget[d];
@@ -201,8 +213,10 @@ int build_layout(sq_ctx* c, cudaStream_t st) {
     if (h2o) off = align_up(off + U * ld.cap * 4);
     ld.victim_off = (long long)off;
     off = align_up(off + U * 4);
-    ld.logit_off = (long long)lfl;
-    if (h2o) lfl += U * ld.cap * G;
+    ld.lse_off = (long long)lse;
+    if (h2o) lse += U * G;
+    ld.logit_off = (long long)(c->wl.lse_floats + lfl);
+    if (slot_logits) lfl += U * ld.cap * G;
   }
   if (off > c->pool_bytes) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the cache pool");
   if (lfl > c->wl.logits_floats) return fail(c, SQ_ERR_CAPACITY, "budgets do not fit the workspace");
@@ -592,6 +606,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.layers = ws_ptr<LayerDesc>(c, c->wl.layers);
     a.pool = c->pool;
     a.logits = ws_ptr<float>(c, c->wl.logits);
+    a.has_logits = c->wl.logits_floats > 0 ? 1 : 0;
     a.part_stat = ws_ptr<float>(c, c->wl.part_stat);
     a.part_o = ws_ptr<float>(c, c->wl.part_o);
     a.q = static_cast<const char*>(q) + (size_t)(s - layer_begin) * q_layer;

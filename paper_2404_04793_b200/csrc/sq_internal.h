@@ -13,10 +13,11 @@ constexpr int kMaxGroup = 128;          // query heads per KV head
 constexpr int kTargetItems = 148 * 16;  // room for split-K pieces beyond one per (layer, unit)
 
 // Per-layer cache geometry, resident in device memory once the budgets are known.
-// k/v/pos/acc/victim offsets are BYTES from the pool base; logit_off counts floats from the
+// k/v/pos/acc/victim offsets are BYTES from the pool base; logit_off and lse_off count floats from the
 // start of the logits area of the workspace.
 struct LayerDesc {
   long long k_off, v_off, pos_off, acc_off, victim_off, logit_off;
+  long long lse_off;      // H2O: [unit][group] row log-sum-exps for the score pass of wide groups
   int b;                  // budget: tokens kept per unit
   int cap;                // slots per unit (b rounded up to page_tokens)
   int b_heavy, b_recent;  // H2O split of b
@@ -90,6 +91,7 @@ struct DecodeArgsBase {
   int n_unit;  // batch * n_kv_head
   int split_tokens, policy;
   int uniform;  // every descriptor of the launch has n_unit items (no split-K): items are found in O(1)
+  int has_logits;  // H2O: the workspace holds the per-slot logits the kernels other than the tcgen05 pair need
   float scale_log2;  // log2(e) / sqrt(head_dim)
 };
 // With split-K: items before the k-th descriptor of the launch (k <= n_layer_total <= kMaxLayers).
@@ -129,5 +131,6 @@ cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_
 cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
 cudaError_t launch_decode_attn_mma(const DecodeArgs& a, int n_items, cudaStream_t s);
 cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s);
+int decode_path_override();  // SQ_DECODE_PATH: 0 none, 1 alu, 2 mma
 
 }  // namespace sq
