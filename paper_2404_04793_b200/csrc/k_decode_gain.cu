@@ -41,9 +41,10 @@ struct Candidate {
 
 // SETS: groups of four token warps (tile i goes to set i % SETS); TMEM_COLS: tensor-memory columns of the CTA
 // (256: three buffers of up to 80 head columns or two of up to 128; 128: one buffer); CTAS: CTAs per SM aimed at.
-template <int STAGES, int SETS, int TMEM_COLS, int CTAS>
+// UNIFORM / Args: 1 / DecodeArgsBase for launches without split-K (no lookup-table search compiled in), else 0 / DecodeArgs.
+template <int STAGES, int SETS, int TMEM_COLS, int CTAS, int UNIFORM, class Args>
 __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
-    h2o_gain_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, DecodeArgs a,
+    h2o_gain_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, Args a,
                        int n_cols, int n_buf) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   Candidate* s_cand = reinterpret_cast<Candidate*>(s_nlse + kTM);          // one per token warp
 
   ItemLoc it;
-  if (!locate(a, blockIdx.x, it)) return;
+  if (!locate<UNIFORM, Args>(a, blockIdx.x, it)) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const LayerDesc* ldp = a.layers + it.layer;
   const int b = ldp->b, cap = ldp->cap, G = a.group;
@@ -262,17 +263,21 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   Candidate best = s_cand[0];
   for (int q = 1; q < 4 * SETS; ++q)
     if (s_cand[q].rank < best.rank) best = s_cand[q];
-  int* victim = reinterpret_cast<int*>(a.pool + ldp->victim_off) + unit;
+  // looked up again rather than carried through the token loop: the registers are needed there
+  if (!locate<UNIFORM, Args>(a, blockIdx.x, it)) return;
+  const LayerDesc* ldt = a.layers + it.layer;
+  const int unit_t = it.local / it.n_split, split_t = it.local - unit_t * it.n_split;
+  int* victim = reinterpret_cast<int*>(a.pool + ldt->victim_off) + unit_t;
   if (it.n_split == 1) {
     *victim = best.slot;
     return;
   }
   // split-K: park this piece's candidate where its attention partials were, take a ticket
-  Candidate* parked = reinterpret_cast<Candidate*>(a.part_stat + ((size_t)it.base + (size_t)unit * it.n_split) * G * kStatStride);
-  const size_t stride = (size_t)G * kStatStride * sizeof(float) / sizeof(Candidate);
-  parked[split * stride] = best;
+  Candidate* parked = reinterpret_cast<Candidate*>(a.part_stat + ((size_t)it.base + (size_t)unit_t * it.n_split) * a.group * kStatStride);
+  const size_t stride = (size_t)a.group * kStatStride * sizeof(float) / sizeof(Candidate);
+  parked[split_t * stride] = best;
   __threadfence();
-  int* ticket = a.tickets + (size_t)it.layer * a.n_unit + unit;
+  int* ticket = a.tickets + (size_t)it.layer * a.n_unit + unit_t;
   if (atomicAdd(ticket, 1) != it.n_split - 1) return;
   __threadfence();
   *ticket = 0;
@@ -300,14 +305,18 @@ cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_byt
     return cudaErrorNotSupported;
   constexpr int kStages = 4, kSets = 2, kTmemCols = 256;
   constexpr size_t smem = 1024 + (size_t)kTM * 128 + (size_t)kStages * kTileBytes + 18 * 8 + kTM * 4 + 8 * sizeof(Candidate);
-  auto kern = h2o_gain_tc_kernel<kStages, kSets, kTmemCols, 2>;
+  auto kern_u = h2o_gain_tc_kernel<kStages, kSets, kTmemCols, 2, 1, DecodeArgsBase>;
+  auto kern_s = h2o_gain_tc_kernel<kStages, kSets, kTmemCols, 2, 0, DecodeArgs>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(kern_u, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern_s, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<n_items, 64 + 128 * kSets, smem, s>>>(tm_q, tm_k, a, n_cols, kTmemCols == 128 ? 1 : (3 * n_cols <= kTmemCols ? 3 : 2));
+  const int n_buf = kTmemCols == 128 ? 1 : (3 * n_cols <= kTmemCols ? 3 : 2);
+  if (a.uniform) kern_u<<<n_items, 64 + 128 * kSets, smem, s>>>(tm_q, tm_k, a, n_cols, n_buf);  // sliced: no table
+  else kern_s<<<n_items, 64 + 128 * kSets, smem, s>>>(tm_q, tm_k, a, n_cols, n_buf);
   return cudaGetLastError();
 }
 
