@@ -78,9 +78,6 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
   const int* pos = reinterpret_cast<const int*>(a.pool + ldp->pos_off) + (size_t)unit * cap;
   float* acc = reinterpret_cast<float*>(a.pool + ldp->acc_off) + (size_t)unit * cap;
-  const float* lse = a.logits + ldp->lse_off + (size_t)unit * G;
-  const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
-  const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
 
   if (tid == 0) {
     mbar_init(bar_q, 1);
@@ -102,6 +99,7 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   }
   if (tid >= 64 && tid < 64 + kTM) {
     const int h = tid - 64;
+    const float* lse = a.logits + ldp->lse_off + (size_t)unit * G;
     // columns past the group read +inf here, so their weight is exp2(-inf) = 0
     s_nlse[h] = (h < G) ? -lse[h] : -INFINITY;
   }
@@ -113,6 +111,9 @@ __global__ void __launch_bounds__(64 + 128 * SETS, CTAS)
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
+      // rows of this unit in the [rows][64] views of the pool and of q (tensor maps)
+      const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
+      const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
       mbar_expect_tx(bar_q, n_cols * 128);
       tma_load_2d(s_u32(q_s), &tm_q, 0, (int)q_row0, bar_q);
       int issued = 0;
