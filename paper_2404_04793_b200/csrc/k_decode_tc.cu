@@ -85,24 +85,16 @@ __global__ void __launch_bounds__(192, 2)
   const int seq = unit / a.n_kv_head, kvh = unit - seq * a.n_kv_head;
   const size_t tok = (size_t)(it.layer - a.layer_begin) * a.batch + seq;
   using bf16 = __nv_bfloat16;
-  bf16* Kb = reinterpret_cast<bf16*>(a.pool + ldp->k_off) + (size_t)unit * cap * kD;
-  bf16* Vb = reinterpret_cast<bf16*>(a.pool + ldp->v_off) + (size_t)unit * cap * kD;
-  const bf16* kn = reinterpret_cast<const bf16*>(a.k_new) + (tok * a.n_kv_head + kvh) * kD;
-  const bf16* vn = reinterpret_cast<const bf16*>(a.v_new) + (tok * a.n_kv_head + kvh) * kD;
-  bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
-  // H2O: the unit's row log-sum-exps (log2 domain), read by the score-update pass that follows
-  float* lse = a.logits + ldp->lse_off + (size_t)unit * G;
-  float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
-  float* po = a.part_o + (size_t)blockIdx.x * G * kD;
-  // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q
-  const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
-  const long long v_row0 = ldp->v_off / (kD * 2) + (long long)unit * cap;
-  const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
+  // (pointers are formed where they are used: the softmax loop needs the registers)
 
   // the CTA whose range holds slot w stores the new token first (generic proxy), then lets
   // the TMA reads (async proxy) see it
   if (w >= t0 && w < t1) {
     if (tid < 16) {
+      bf16* Kb = reinterpret_cast<bf16*>(a.pool + ldp->k_off) + (size_t)unit * cap * kD;
+      bf16* Vb = reinterpret_cast<bf16*>(a.pool + ldp->v_off) + (size_t)unit * cap * kD;
+      const bf16* kn = reinterpret_cast<const bf16*>(a.k_new) + (tok * a.n_kv_head + kvh) * kD;
+      const bf16* vn = reinterpret_cast<const bf16*>(a.v_new) + (tok * a.n_kv_head + kvh) * kD;
       const bool is_v = tid >= 8;
       const int c = tid & 7;
       const uint4 val = *reinterpret_cast<const uint4*>((is_v ? vn : kn) + c * 8);
@@ -142,6 +134,10 @@ __global__ void __launch_bounds__(192, 2)
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
+      // rows of this unit in the [rows][64] views of the pool (tensor maps) and of q
+      const long long k_row0 = ldp->k_off / (kD * 2) + (long long)unit * cap;
+      const long long v_row0 = ldp->v_off / (kD * 2) + (long long)unit * cap;
+      const long long q_row0 = (long long)(tok * a.n_q_head + (size_t)kvh * G);
       mbar_expect_tx(bar_q, kQBytes);
       tma_load_2d(s_u32(q_s), &tm_q, 0, (int)q_row0, bar_q);
       int issued = 0;
@@ -328,6 +324,9 @@ __global__ void __launch_bounds__(192, 2)
     if (ok) ok = mbar_wait(bar_odone, (n_tiles - 1) & 1, abort_flag);
     if (ok && warp_live) {
       tc_fence_after();
+      bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
+      float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
+      float* po = a.part_o + (size_t)blockIdx.x * G * kD;
       const float inv = 1.f / l_w;
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
@@ -351,7 +350,8 @@ __global__ void __launch_bounds__(192, 2)
         stat[row * kStatStride] = m_ref;
         stat[row * kStatStride + 1] = H2O ? l_true : l_w;
         stat[row * kStatStride + 2] = l_w;
-        if (H2O && it.n_split == 1) lse[row] = m_ref + log2f(l_true);
+        // H2O: the unit's row log-sum-exps (log2 domain), read by the score-update pass that follows
+        if (H2O && it.n_split == 1) (a.logits + ldp->lse_off + (size_t)unit * G)[row] = m_ref + log2f(l_true);
       }
     }
   }
@@ -362,7 +362,7 @@ __global__ void __launch_bounds__(192, 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicOr(a.status, kStatusTimeout);
-  if (it.n_split > 1) merge_if_last<bf16>(a, it, unit, H2O ? lse : nullptr);
+  if (it.n_split > 1) merge_if_last<bf16>(a, it, unit, H2O ? a.logits + ldp->lse_off + (size_t)unit * G : nullptr);
 }
 
 template <int STAGES, int ROWS, bool H2O>
