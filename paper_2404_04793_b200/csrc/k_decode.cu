@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(128, GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) dec
 // each kept token's probabilities (summed over the group's heads in head order) to its score
 // and picks the slot the next append replaces.
 template <typename T>
-__global__ void __launch_bounds__(kSelThreads) decode_combine_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(kSelThreads, 5) decode_combine_kernel(DecodeArgs a) {
   __shared__ SelScratch sc;
   __shared__ __align__(16) float s_M[kMaxGroup], s_invL[kMaxGroup], s_invLw[kMaxGroup];
   // one CTA per (descriptor of the launch, unit)
