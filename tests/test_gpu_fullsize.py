@@ -92,3 +92,39 @@ def test_falcon_7b_mqa_cells():
 def test_falcon_7b_largest_cell_sampled():
     # the largest cell of the sweep: batch 224, prompt 16384, budget 50 % (15 GB of K/V per step)
     _follow(synth.falcon_7b(224, 16384, 50.0, synth.SLIDING_WINDOW), n_units=36, steps=2)
+
+
+def test_llama2_7b_per_sequence_budgets_full_size():
+    """The benchmark shape with one budget vector per sequence (the batch's vector rotated by one
+    layer per sequence, so every sequence differs and every vector sums to n_layer * b_init)."""
+    w = synth.llama2_7b().replace(steps=8)
+    base, _ = O.allocate_budgets(np.array(synth.cos_targets(w.n_layer), dtype=np.float32), w.b_init, w.p)
+    base = base.tolist()
+    rows = [base[s:] + base[:s] for s in range(w.batch)]
+    ctx = engine.context_for(w, DEV, per_sequence_budgets=1)
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets(rows)
+    assert ctx.get_budgets()[0] == rows
+    units = H.sample_units(w, 40, seed=3)
+    by_layer = {}
+    for u in units:
+        by_layer.setdefault(u[0], []).append(u)
+    oracles = {}
+    for l in range(w.n_layer):
+        _, k, v = synth.prompt_qkv(w, l, DEV, need_q=False)
+        ctx.prefill_compress(l, k, v)
+        for (_, s, h) in by_layer.get(l, []):
+            u = O.UnitCache(w.policy, rows[s][l], w.n_sink, w.heavy_num, w.heavy_den)
+            u.prefill(H.f64(k[s, h]), H.f64(v[s, h]), None)
+            oracles[(l, s, h)] = u
+        del k, v
+    for t in range(w.steps):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+        for (l, s, h), u in oracles.items():
+            want = u.decode_step(H.f64(q[l, s, h:h + 1]), H.f64(kn[l, s, h]), H.f64(vn[l, s, h]))
+            assert np.max(np.abs(H.f64(out[l, s, h:h + 1]) - want)) <= H.TOL_OUT[w.dtype], (t, l, s, h)
+    for key, u in oracles.items():
+        assert ctx.get_kept(*key)[0] == u.kept_positions(), key
+    assert ctx.status() == 0
