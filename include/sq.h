@@ -122,8 +122,9 @@ int sq_layer_importance(sq_ctx* ctx, int32_t layer, const void* hidden_in, const
  * 1 <= b_init <= the b_init of sq_ctx_create.  Runs on the device. */
 int sq_allocate_budgets(sq_ctx* ctx, int64_t b_init, double p, void* stream);
 
-/* Sets the per-layer budgets directly (host array [n_layer]), bypassing importance and
- * clustering.  SQ_ERR_CAPACITY if they do not fit the pool. */
+/* Sets the per-layer budgets directly (host array [n_layer]; [batch][n_layer] with
+ * per_sequence_budgets), bypassing importance and clustering.  SQ_ERR_CAPACITY if they do not
+ * fit the pool. */
 int sq_set_budgets(sq_ctx* ctx, const int32_t* budgets_host, void* stream);
 
 /* Algorithm 1, step 13, with the first compression (steps 16-18) applied at once: caches the
@@ -152,22 +153,24 @@ int sq_decode_step(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, const vo
                    const void* v_new, void* out, void* stream);
 
 /* C_seq(K, b) on its own (Section 4.1): lowers the budgets of layers [layer_begin, layer_end)
- * to new_budgets_host[i] (host array, each <= the layer's current budget, >= 1) and compresses
- * their caches in place to at most that many tokens. */
+ * to new_budgets_host[i] (host array [layer_end-layer_begin], or [batch][layer_end-layer_begin]
+ * with per_sequence_budgets; each <= the current budget, >= 1) and compresses their caches in
+ * place to at most that many tokens.  One kernel launch serves all layers of the call. */
 int sq_evict(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, const int32_t* new_budgets_host,
              void* stream);
 
 /* Read-back (host outputs; these synchronise). */
-int sq_get_cos_sim(sq_ctx* ctx, float* cos_sim_host /* [n_layer] */);
-int sq_get_budgets(sq_ctx* ctx, int32_t* budgets_host /* [n_layer] */, uint8_t* is_g3_host /* [n_layer] or NULL */);
+int sq_get_cos_sim(sq_ctx* ctx, float* cos_sim_host /* [n_layer]; [batch][n_layer] with per_sequence_budgets */);
+int sq_get_budgets(sq_ctx* ctx, int32_t* budgets_host /* same shape */, uint8_t* is_g3_host /* same shape, or NULL */);
 /* Kept tokens of one unit, sorted by position: positions and (H2O; else zeros) scores.
- * Arrays must hold budget[layer] entries; *n receives the count. */
+ * Arrays must hold the unit's budget (sq_get_len(layer) entries always suffice); *n receives
+ * the count. */
 int sq_get_kept(sq_ctx* ctx, int32_t layer, int32_t seq, int32_t kv_head, int32_t* pos_host, float* acc_host,
                 int32_t* n);
 /* Cached K and V rows of one unit in the same (position) order as sq_get_kept, as raw
  * elements of the context's dtype: [n, head_dim] each (host buffers). */
 int sq_get_kv(sq_ctx* ctx, int32_t layer, int32_t seq, int32_t kv_head, void* k_host, void* v_host);
-/* Number of cached tokens per unit of a layer. */
+/* Number of cached tokens per unit of a layer (with per_sequence_budgets: of its longest unit). */
 int sq_get_len(sq_ctx* ctx, int32_t layer, int32_t* len);
 /* Device-side status word: 0 = clean; non-zero = a kernel detected an inconsistency. */
 int sq_status(sq_ctx* ctx, int32_t* device_status);
