@@ -209,7 +209,6 @@ int sq_kv_bytes_per_step(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, in
 int sq_prompt_scores_static(const void* q_prompt, const void* k_prompt, int32_t batch, int32_t n_q_head,
                             int32_t n_kv_head, int32_t prompt_len, int32_t head_dim, int32_t dtype, float* acc_out,
                             void* stream);
-int64_t sq_prompt_scores_static_max_rows(void);
 
 #ifdef __cplusplus
 }

@@ -18,6 +18,7 @@ LIB_PATH = os.environ.get("SQ_LIB_PATH") or os.path.join(_PKG, "libsq.so")
 SQ_OK, SQ_ERR_INVALID_ARG, SQ_ERR_STATE, SQ_ERR_CAPACITY, SQ_ERR_CUDA, SQ_ERR_UNSUPPORTED = range(6)
 SQ_POLICY_SLIDING_WINDOW, SQ_POLICY_STREAMING_LLM, SQ_POLICY_H2O = 0, 1, 2
 SQ_F32, SQ_BF16 = 0, 1
+SQ_STATIC_SCORE_MAX_ROWS = 1 << 20  # mirrors include/sq.h
 _ERR_NAMES = {1: "SQ_ERR_INVALID_ARG", 2: "SQ_ERR_STATE", 3: "SQ_ERR_CAPACITY", 4: "SQ_ERR_CUDA",
               5: "SQ_ERR_UNSUPPORTED"}
 
@@ -25,8 +26,7 @@ _ERR_NAMES = {1: "SQ_ERR_INVALID_ARG", 2: "SQ_ERR_STATE", 3: "SQ_ERR_CAPACITY", 
 EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequence_batch",
            "sq_layer_importance", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
            "sq_decode_step", "sq_evict", "sq_get_cos_sim", "sq_get_budgets", "sq_get_kept", "sq_get_kv",
-           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static",
-           "sq_prompt_scores_static_max_rows"]
+           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static"]
 
 
 class sq_config(ctypes.Structure):
@@ -75,10 +75,8 @@ def lib() -> ctypes.CDLL:
     L.sq_last_error.restype = c_char_p
     L.sq_kv_bytes_per_step.argtypes = [P, c_int32, c_int32, POINTER(c_int64)]
     L.sq_prompt_scores_static.argtypes = [P, P, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, P, P]
-    L.sq_prompt_scores_static_max_rows.argtypes = []
-    L.sq_prompt_scores_static_max_rows.restype = c_int64
     for name in EXPORTS:
-        if name not in ("sq_last_error", "sq_prompt_scores_static_max_rows"):
+        if name != "sq_last_error":
             getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L

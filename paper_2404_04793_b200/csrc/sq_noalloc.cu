@@ -56,5 +56,3 @@ extern "C" int sq_prompt_scores_static(const void* q_prompt, const void* k_promp
   if (sq::launch_prefill_scores_alu(a, dtype, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SQ_ERR_CUDA;
   return SQ_OK;
 }
-
-extern "C" int64_t sq_prompt_scores_static_max_rows(void) { return kMaxRows; }

@@ -53,8 +53,7 @@ def test_static_scores_match_regular_entry_point_twice_in_a_row():
 
 
 def test_static_scores_reject_oversized_and_bad_requests():
-    cap = B.lib().sq_prompt_scores_static_max_rows()
-    assert cap == 1 << 20
+    cap = B.SQ_STATIC_SCORE_MAX_ROWS
     q = torch.zeros(1, 2, 8, 64, device=DEV)
     k = torch.zeros(1, 1, 8, 64, device=DEV)
     acc = torch.zeros(1, 1, 8, device=DEV)
