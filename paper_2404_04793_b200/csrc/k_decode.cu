@@ -337,6 +337,111 @@ __global__ void __launch_bounds__(kSelThreads, 5) decode_combine_kernel(DecodeAr
   }
 }
 
+// H2O bookkeeping for launches without split-K and groups of at most 32 heads: one WARP per
+// (descriptor, unit) instead of one CTA.  A unit holds a few hundred to a few thousand slots,
+// too little to occupy 256 threads for longer than the block's set-up and reductions take; as
+// warps, every unit of a step is resident at once and nothing synchronises beyond a warp.
+// The arithmetic per slot (head order of the sum, the reciprocal of the row sum) is that of
+// decode_combine_kernel, so both give the same bits.
+constexpr int kWarpUpdWarps = 8;
+__global__ void __launch_bounds__(32 * kWarpUpdWarps, 3) h2o_update_warp_kernel(DecodeArgsBase a) {
+  __shared__ __align__(16) float s_M[kWarpUpdWarps][32], s_invL[kWarpUpdWarps][32];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int idx = blockIdx.x * kWarpUpdWarps + wib;
+  if (idx >= a.n_layer_total * a.n_unit) return;
+  const int k = idx / a.n_unit, unit = idx - k * a.n_unit;
+  const int layer = a.order[k], G = a.group;
+  const LayerDesc* ldp = a.layers + layer;
+  const int b = ldp->b, cap = ldp->cap;
+  const float* stat = a.part_stat + ((size_t)k * a.n_unit + unit) * G * kStatStride;
+  if (lane < G) {
+    const float2 ml = *reinterpret_cast<const float2*>(stat + lane * kStatStride);
+    s_M[wib][lane] = ml.x;
+    s_invL[wib][lane] = 1.f / ml.y;
+  }
+  __syncwarp();
+  const float* wM = s_M[wib];
+  const float* wI = s_invL[wib];
+  const int len = min(a.n_tok + 1, b);
+  const bool full = (len == b);
+  const int thr = a.n_tok + 1 - ldp->b_recent;  // next step: positions <= thr are outside the recent window
+  const int* pos = reinterpret_cast<const int*>(a.pool + ldp->pos_off) + (size_t)unit * cap;
+  float* acc = reinterpret_cast<float*>(a.pool + ldp->acc_off) + (size_t)unit * cap;
+  const float* logit = a.logits + ldp->logit_off + (size_t)unit * cap * G;
+  unsigned long long best = ~0ull;
+  int best_slot = -1;
+  constexpr int kIl = 8;  // slots per lane in flight: their logits, score and position loads are independent
+  for (int s0 = lane; s0 < len; s0 += kIl * 32) {
+    float gain[kIl], old[kIl];
+    int p[kIl];
+#pragma unroll
+    for (int u = 0; u < kIl; ++u) {
+      const int slot = s0 + u * 32;
+      gain[u] = 0.f;
+      old[u] = 0.f;
+      p[u] = 0x7fffffff;
+      if (slot < len) {
+        old[u] = acc[slot];
+        if (full) p[u] = pos[slot];
+      }
+    }
+    if ((G & 3) == 0) {
+      for (int h = 0; h < G; h += 4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(wM + h), i4 = *reinterpret_cast<const float4*>(wI + h);
+        float4 l4[kIl];
+#pragma unroll
+        for (int u = 0; u < kIl; ++u) {
+          const int slot = s0 + u * 32;
+          l4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (slot < len) l4[u] = *reinterpret_cast<const float4*>(logit + (size_t)slot * G + h);
+        }
+#pragma unroll
+        for (int u = 0; u < kIl; ++u) {
+          gain[u] += exp2f(l4[u].x - m4.x) * i4.x;
+          gain[u] += exp2f(l4[u].y - m4.y) * i4.y;
+          gain[u] += exp2f(l4[u].z - m4.z) * i4.z;
+          gain[u] += exp2f(l4[u].w - m4.w) * i4.w;
+        }
+      }
+    } else {
+#pragma unroll 1
+      for (int u = 0; u < kIl; ++u) {
+        const int slot = s0 + u * 32;
+        if (slot >= len) continue;
+        float g1 = 0.f;
+        for (int h = 0; h < G; ++h) g1 += exp2f(logit[(size_t)slot * G + h] - wM[h]) * wI[h];
+        gain[u] = g1;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kIl; ++u) {
+      const int slot = s0 + u * 32;
+      if (slot >= len) continue;
+      const float v = old[u] + gain[u];
+      acc[slot] = v;
+      if (full && p[u] <= thr) {
+        const unsigned long long r = victim_rank(v, p[u]);
+        if (r < best) {
+          best = r;
+          best_slot = slot;
+        }
+      }
+    }
+  }
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long c2 = __shfl_xor_sync(kFull, best, o);
+      const int s2 = __shfl_xor_sync(kFull, best_slot, o);
+      if (c2 < best) {
+        best = c2;
+        best_slot = s2;
+      }
+    }
+    if (lane == 0) reinterpret_cast<int*>(a.pool + ldp->victim_off)[unit] = best_slot;
+  }
+}
+
 template <typename T, int D>
 static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
   if (a.group == 1) {
@@ -360,6 +465,17 @@ int decode_path_override() {
     mode = !e ? 0 : (!strcmp(e, "alu") ? 1 : (!strcmp(e, "mma") ? 2 : 0));
   }
   return mode;
+}
+
+// SQ_H2O_UPDATE=cta keeps the H2O score update of unsplit launches on the CTA-per-unit kernel
+// (for A/B measurements).
+static bool h2o_update_override() {
+  static int mode = -1;
+  if (mode < 0) {
+    const char* e = getenv("SQ_H2O_UPDATE");
+    mode = (e && !strcmp(e, "cta")) ? 1 : 0;
+  }
+  return mode == 1;
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
@@ -397,6 +513,13 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || !need_combine) return e;
   const int n_cta = a.n_layer_total * a.n_unit;
+  // More units than the CTA-per-unit kernel holds in one wave (5 CTAs per SM), and nothing to
+  // merge: only the scores and the next victim remain, one warp per unit.  Smaller launches
+  // (one layer of a small batch) finish sooner with a CTA per unit.
+  if (a.policy == SQ_POLICY_H2O && a.uniform && a.group <= 32 && n_cta > 148 * 5 && !h2o_update_override()) {
+    h2o_update_warp_kernel<<<(n_cta + kWarpUpdWarps - 1) / kWarpUpdWarps, 32 * kWarpUpdWarps, 0, s>>>(a);
+    return cudaGetLastError();
+  }
   if (dtype == SQ_F32)
     decode_combine_kernel<float><<<n_cta, kSelThreads, 0, s>>>(a);
   else
