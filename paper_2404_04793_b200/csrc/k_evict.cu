@@ -4,10 +4,16 @@
 //      over the scores) and record the decisions as a bitmask in shared memory with a running
 //      count per 32 slots, so that any thread knows a row's new slot without touching memory;
 //   2. close the gaps by moving the kept rows towards slot 0 in slot order.  A row's new slot
-//      is never behind its old one, so reads may run ahead of writes freely: chunks of rows
-//      stream through a multi-stage cp.async ring (rows, positions and scores alike) and are
-//      stored to their new slots when they land.  Only the store of a chunk must follow the
-//      loads of the chunks before it, which the ring order guarantees.
+//      is never behind its old one, so a chunk of rows (with its positions and scores) is
+//      fetched into shared memory with cp.async and stored to its new slots once it has
+//      landed; chunks go in slot order, so a store never overwrites a row not yet read.
+// The kernel is templated on the chunk size and on the number of chunks in flight per CTA.
+// Measured (budgets halved on full caches, GB/s of rows read + written, Llama-2-7B- /
+// Mistral-7B-H2O- / Llama-2-70B-shaped): 32 KB x 3 in flight (2 CTAs per SM) 2837 / 1868 / 3343;
+// 16 KB x 3: 3727 / 2573 / 4513; 8 KB x 4: 3812 / 2776 / 4582; 16 KB x 2: 4180 / 2947 / 4901;
+// 16 KB x 1: 4148 / 2987 / 5024; 32 KB x 1 (7 CTAs per SM): 4176 / 2982 / 5124.  The overlap
+// that matters comes from many resident CTAs, not from a deep ring inside one, so the build
+// uses one 32 KB chunk per CTA.
 #include "sq_device.cuh"
 #include "sq_internal.h"
 #include "sq_select.cuh"
@@ -15,10 +21,7 @@
 namespace sq {
 
 namespace {
-constexpr int kChunkBytes = 32 * 1024;  // K and V rows of one chunk
-constexpr int kStages = 3;              // 96 KB of rows in flight per CTA, two CTAs per SM
 constexpr int kMaxVecPerRow = 32;       // 512-byte rows (fp32, head_dim 128)
-constexpr int kMaxChunkRows = kChunkBytes / (2 * 128);  // 128-byte rows (bf16, head_dim 64)
 
 __device__ __forceinline__ void cp_async(void* dst_smem, const void* src, int bytes16) {
   const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst_smem);
@@ -32,14 +35,19 @@ __device__ __forceinline__ void cp_async_wait_all_but(int n) {
   switch (n) {
     case 0: asm volatile("cp.async.wait_group 0;"); break;
     case 1: asm volatile("cp.async.wait_group 1;"); break;
-    default: asm volatile("cp.async.wait_group 2;"); break;
+    case 2: asm volatile("cp.async.wait_group 2;"); break;
+    case 3: asm volatile("cp.async.wait_group 3;"); break;
+    case 4: asm volatile("cp.async.wait_group 4;"); break;
+    default: asm volatile("cp.async.wait_group 5;"); break;
   }
 }
 }  // namespace
 
 // Dynamic shared memory: kStages chunks of rows, then per stage the chunk's positions and
 // scores, then the keep bitmask (one word per 32 slots) and its running count.
+template <int kChunkBytes, int kStages>
 __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
+  constexpr int kMaxChunkRows = kChunkBytes / (2 * 128);  // 128-byte rows (bf16, head_dim 64)
   extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ SelScratch sc;
   uint4* stage = reinterpret_cast<uint4*>(dyn);
@@ -152,8 +160,17 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
     }
     cp_async_commit();  // one group per chunk, empty past the end, so the wait counts stay aligned
   };
-  for (int c = 0; c < kStages - 1; ++c) issue(c);
-  for (int c = 0; c < n_chunks; ++c) {
+  // chunks before the first kept row that moves hold nothing to do
+  int c_begin = n_chunks;
+  for (int w = 0; w < n_words; ++w) {
+    const unsigned m = s_mask[w];
+    if (s_before[w] + __popc(m) != (w + 1) * 32 || w == n_words - 1) {  // first word with a gap (or the last)
+      c_begin = (w * 32) / rows;
+      break;
+    }
+  }
+  for (int c = c_begin; c < c_begin + kStages - 1; ++c) issue(c);
+  for (int c = c_begin; c < n_chunks; ++c) {
     issue(c + kStages - 1);
     cp_async_wait_all_but(kStages - 1);
     __syncthreads();
@@ -199,20 +216,27 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
   }
 }
 
-cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s) {
-  if (a.row_bytes / 16 > kMaxVecPerRow || a.row_bytes < 128 || (a.row_bytes & (a.row_bytes - 1)))
-    return cudaErrorInvalidValue;
+template <int kChunkBytes, int kStages>
+static cudaError_t launch_evict_cfg(const EvictArgs& a, cudaStream_t s) {
+  constexpr int kMaxChunkRows = kChunkBytes / (2 * 128);
   const size_t words = ((size_t)a.max_cap + 31) / 32;
   const size_t smem = (size_t)kStages * kChunkBytes + (size_t)kStages * kMaxChunkRows * 8 + words * 8;
   if (smem > 200 * 1024) return cudaErrorInvalidValue;  // caches beyond ~1.4 M slots per unit
   static size_t configured = 0;
   if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(evict_kernel<kChunkBytes, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  evict_kernel<<<dim3(a.n_unit, a.n_layers), kSelThreads, smem, s>>>(a);
+  evict_kernel<kChunkBytes, kStages><<<dim3(a.n_unit, a.n_layers), kSelThreads, smem, s>>>(a);
   return cudaGetLastError();
+}
+
+cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s) {
+  if (a.row_bytes / 16 > kMaxVecPerRow || a.row_bytes < 128 || (a.row_bytes & (a.row_bytes - 1)))
+    return cudaErrorInvalidValue;
+  return launch_evict_cfg<32 * 1024, 1>(a, s);
 }
 
 }  // namespace sq

@@ -49,16 +49,40 @@ __device__ uint32_t block_radix_select(SelScratch& sc, int n, unsigned int k, Ke
       if ((kk & mask) == prefix) atomicAdd(&sc.hist[(kk >> shift) & 0xffu], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      unsigned int rem = sc.k_rem, above = 0u;
-      int d = 255;
-      for (; d > 0; --d) {
-        if (above + sc.hist[d] >= rem) break;
-        above += sc.hist[d];
+    if (tid < 32) {
+      // The digit is the highest d with (entries in bins above d) + hist[d] >= rem.  Lane l owns
+      // the eight bins 255 - 8l ... 248 - 8l; a warp scan gives the entries above each lane's
+      // bins, and the one lane whose bins hold the crossing walks them.
+      const unsigned int rem = sc.k_rem;
+      unsigned int c[8], sum = 0u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        c[j] = sc.hist[255 - (8 * tid + j)];
+        sum += c[j];
       }
-      sc.k_rem = rem - above;
-      sc.prefix = prefix | ((uint32_t)d << shift);
-      sc.total = sc.hist[d];
+      unsigned int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (tid >= o) incl += t;
+      }
+      unsigned int above = incl - sum;
+      const bool here = (above < rem) && (incl >= rem);
+      const bool none = (__ballot_sync(0xffffffffu, here) == 0u);  // rem beyond the set: digit 0, as a serial walk ends
+      if (here || (none && tid == 31)) {
+        int j = 0;
+        for (; j < 7; ++j) {
+          if (above + c[j] >= rem) break;
+          above += c[j];
+        }
+        if (none) {  // lane 31: bins 7..0, the walk stops at bin 0 with everything above it counted
+          j = 7;
+          above = incl - c[7];
+        }
+        sc.k_rem = rem - above;
+        sc.prefix = prefix | ((uint32_t)(255 - (8 * tid + j)) << shift);
+        sc.total = c[j];
+      }
     }
     __syncthreads();
   }

@@ -160,6 +160,45 @@ def touch_all_kernels(w: synth.Workload, device="cuda:0"):
     return dict(workload=w.name, what="every kernel once", budgets=budgets, device_status=ctx.status())
 
 
+def evict_time(w: synth.Workload, reps=3, device="cuda:0"):
+    """Times one explicit eviction (sq_evict over all layers, budgets halved) on caches filled to
+    their budgets; the context is refilled before every repetition, since an eviction is not
+    repeatable.  Algorithmic bytes: the rows that stay, read and written once each (K and V,
+    positions, and scores for H2O)."""
+    job = engine.Job(w.replace(steps=1), device)
+    ctx = job.ctx
+    g = torch.Generator(device=device).manual_seed(1)
+    shape_kv = (w.batch, w.n_kv_head, w.prompt, w.head_dim)
+    k = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    v = torch.randn(shape_kv, generator=g, device=device).to(w.dtype)
+    acc = torch.rand(w.batch, w.n_kv_head, w.prompt, generator=g, device=device) if w.policy == synth.H2O else None
+    floor = (w.n_sink + 1) if w.policy == synth.STREAMING_LLM else 1
+    times = []
+    for _ in range(reps + 1):
+        ctx.begin_sequence_batch(w.batch, w.prompt)
+        for l in range(w.n_layer):
+            a, b = synth.hidden_pair(w, l, device, batch=1, n_tok=256)
+            ctx.layer_importance(l, a, b)
+        ctx.allocate_budgets(w.b_init, w.p)
+        budgets, _ = ctx.get_budgets()
+        for l in range(w.n_layer):
+            ctx.prefill_compress(l, k, v, None, acc)
+        new = [max(floor, b // 2) for b in budgets]
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.evict(0, w.n_layer, new)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = min(times[1:])
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    per_row = 2 * w.head_dim * e + 4 + (4 if w.policy == synth.H2O else 0)
+    moved = 2 * w.batch * w.n_kv_head * sum(min(n, min(w.prompt, b)) for n, b in zip(new, budgets)) * per_row
+    return dict(workload=w.name, what="sq_evict, all layers, budgets halved", ms=round(ms, 4), all_ms=[round(t, 4) for t in times],
+                algorithmic_bytes=moved, GBs=round(moved / ms / 1e6, 1), device_status=ctx.status())
+
+
 def generation_throughput(w: synth.Workload, device="cuda:0"):
     """Decode tokens/s of the attention + eviction path over a whole generation: cache filled
     from a prompt of w.prompt tokens, then w.steps fused decode steps, all timed together."""
@@ -234,6 +273,7 @@ def main():
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--per-sequence", action="store_true", help="per-sequence budgets (a rotated budget vector per sequence)")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
+    ap.add_argument("--evict", action="store_true", help="time one explicit eviction of all layers to half the budgets")
     ap.add_argument("--all-kernels", action="store_true", help="launch every kernel of the library once or a few times")
     ap.add_argument("--layers", type=int, default=0, help="with --all-kernels: number of layers of the shape to keep")
     ap.add_argument("--compare-budgets", action="store_true",
@@ -264,6 +304,9 @@ def main():
         return
     if args.prefill:
         print(json.dumps(prefill_compress_time(build_workload(args), args.steps)), flush=True)
+        return
+    if args.evict:
+        print(json.dumps(evict_time(build_workload(args), min(args.steps, 5))), flush=True)
         return
     print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer,
                                       per_sequence=args.per_sequence)), flush=True)
