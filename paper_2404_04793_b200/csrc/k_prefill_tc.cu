@@ -23,9 +23,16 @@ namespace sq {
 
 using namespace tc;
 
+// Threads per CTA: a TMA warp, an MMA warp and eight drain warps.  A warp reaches only the 32
+// tensor-memory lanes of its quarter (warp index mod 4), so each quarter of the accumulator rows
+// is drained by two warps that take 64 of the tile's 128 columns each: four drain warps per
+// scheduler (two CTAs per SM) instead of two, so the special-function pipe is fed while other
+// warps wait for an accumulator or a tensor-memory load.
+constexpr int kPrefillThreads = 64 + 256;
+
 // SWEEP 1: rows = queries, streamed tiles = keys; SWEEP 2: rows = keys, streamed tiles = queries.
 template <int D, int STAGES, int SWEEP>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kPrefillThreads, 2)
     prefill_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_rows, const __grid_constant__ CUtensorMap tm_stream,
                              ScoreArgs a, float scale_log2, int* status) {
   constexpr int SUB = D / 64;                  // 64-column sub-tiles per operand tile
@@ -88,8 +95,8 @@ __global__ void __launch_bounds__(192, 1)
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_sfull(b), 1);
-      mbar_init(bar_sfree(b), 128);
-      mbar_init(bar_lse(b), 128);
+      mbar_init(bar_sfree(b), 256);
+      mbar_init(bar_lse(b), 256);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -155,9 +162,10 @@ __global__ void __launch_bounds__(192, 1)
   } else {
     // ---------------- accumulator drain: thread = one row of the fixed tile ----------------
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;  // which 64 columns of every tile this warp drains
     const int row = quarter * 32 + lane;
     const int row_idx = row_tile * kTM + row;  // query index (sweep 1) / key index (sweep 2)
-    const int t128 = (warp - 2) * 32 + lane;
+    const int t256 = (warp - 2) * 32 + lane;
     float m = -INFINITY, l = 0.f, colsum = 0.f;
     bool ok = true;
     for (int i = 0; ok && i < n_stream; ++i) {
@@ -165,8 +173,10 @@ __global__ void __launch_bounds__(192, 1)
       int h, qt;
       stream_row0(i, h, qt);
       if (SWEEP == 2) {
-        const int q = qt * kTM + t128;
-        lse_s[buf * kTM + t128] = (q < P) ? a.lse2[((size_t)bi * a.n_q_head + hk * g + h) * P + q] : INFINITY;
+        if (t256 < kTM) {
+          const int q = qt * kTM + t256;
+          lse_s[buf * kTM + t256] = (q < P) ? a.lse2[((size_t)bi * a.n_q_head + hk * g + h) * P + q] : INFINITY;
+        }
         mbar_arrive(bar_lse(buf));  // all 128 row sums of this query tile are staged
         ok = mbar_wait(bar_lse(buf), (i >> 1) & 1, abort_flag);
       }
@@ -175,7 +185,7 @@ __global__ void __launch_bounds__(192, 1)
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const bool diag = (qt == row_tile);
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 2 * half; c < 2 * half + 2; ++c) {
         float v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTM + c * 32, v);
         if (SWEEP == 1) {
@@ -217,11 +227,24 @@ __global__ void __launch_bounds__(192, 1)
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(bar_sfree(buf));
     }
-    if (ok && row_idx < P) {
-      if (SWEEP == 1)
-        a.lse2[((size_t)bi * a.n_q_head + hq) * P + row_idx] = m + log2f(l);
-      else
-        a.acc_prompt[((size_t)bi * a.n_kv_head + hk) * P + row_idx] = colsum;
+    // the two halves of a row meet in shared memory (the staging area is free once every drain
+    // thread is past its last tile); every drain thread reaches both barriers, aborted or not
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (half == 1) {
+      lse_s[2 * row] = (SWEEP == 1) ? m : colsum;
+      lse_s[2 * row + 1] = l;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (half == 0 && ok && !*abort_flag && row_idx < P) {
+      const float o0 = lse_s[2 * row], o1 = lse_s[2 * row + 1];
+      if (SWEEP == 1) {
+        // this half holds column 0 of every tile, so m is finite; the other half may be empty
+        const float mm = fmaxf(m, o0);
+        const float ll = l * ex2(m - mm) + o1 * ex2(o0 - mm);
+        a.lse2[((size_t)bi * a.n_q_head + hq) * P + row_idx] = mm + log2f(ll);
+      } else {
+        a.acc_prompt[((size_t)bi * a.n_kv_head + hk) * P + row_idx] = colsum + o0;
+      }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -284,10 +307,10 @@ static cudaError_t launch_tc_t(const ScoreArgs& a, int* status, cudaStream_t s) 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  k1<<<dim3(n_tile, a.n_q_head, a.batch), 192, smem, s>>>(tm_q, tm_k, a, scale_log2, status);
+  k1<<<dim3(n_tile, a.n_q_head, a.batch), kPrefillThreads, smem, s>>>(tm_q, tm_k, a, scale_log2, status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k2<<<dim3(n_tile, a.n_kv_head, a.batch), 192, smem, s>>>(tm_k, tm_q, a, scale_log2, status);
+  k2<<<dim3(n_tile, a.n_kv_head, a.batch), kPrefillThreads, smem, s>>>(tm_k, tm_q, a, scale_log2, status);
   return cudaGetLastError();
 }
 
