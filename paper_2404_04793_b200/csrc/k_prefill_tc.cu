@@ -168,14 +168,24 @@ __global__ void __launch_bounds__(kPrefillThreads, 2)
     const int t256 = (warp - 2) * 32 + lane;
     float m = -INFINITY, l = 0.f, colsum = 0.f;
     bool ok = true;
+    // sweep 2: the row log-sum-exp of query t256 of streamed tile i; fetched one tile ahead, so
+    // that its trip to memory runs under the previous tile's arithmetic
+    auto fetch_lse = [&](int i) -> float {
+      int h, qt;
+      stream_row0(i, h, qt);
+      const int q = qt * kTM + t256;
+      return (q < P) ? a.lse2[((size_t)bi * a.n_q_head + hk * g + h) * P + q] : INFINITY;
+    };
+    float lse_next = 0.f;
+    if (SWEEP == 2 && t256 < kTM && n_stream > 0) lse_next = fetch_lse(0);
     for (int i = 0; ok && i < n_stream; ++i) {
       const int buf = i & 1;
       int h, qt;
       stream_row0(i, h, qt);
       if (SWEEP == 2) {
         if (t256 < kTM) {
-          const int q = qt * kTM + t256;
-          lse_s[buf * kTM + t256] = (q < P) ? a.lse2[((size_t)bi * a.n_q_head + hk * g + h) * P + q] : INFINITY;
+          lse_s[buf * kTM + t256] = lse_next;
+          if (i + 1 < n_stream) lse_next = fetch_lse(i + 1);
         }
         mbar_arrive(bar_lse(buf));  // all 128 row sums of this query tile are staged
         ok = mbar_wait(bar_lse(buf), (i >> 1) & 1, abort_flag);
