@@ -58,19 +58,21 @@ __global__ void __launch_bounds__(kPrefillThreads, 2)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int P = a.prompt, g = a.n_q_head / a.n_kv_head;
   const int n_tile = (P + kTM - 1) / kTM;
-  const int bi = blockIdx.z;
+  // grid = (head, sequence, tile): the tile index varies slowest, so the CTAs with the most streamed
+  // tiles of every head and sequence start first and the short ones fill the tail of the launch
+  const int bi = blockIdx.y;
   int row_tile, n_stream;
   long long rows0;  // first row of this CTA's fixed tile in the rows tensor
   int hq = 0, hk = 0;
   if (SWEEP == 1) {
-    hq = blockIdx.y;
+    hq = blockIdx.x;
     hk = hq / g;
-    row_tile = n_tile - 1 - blockIdx.x;  // longest rows first
+    row_tile = n_tile - 1 - blockIdx.z;  // longest rows first
     n_stream = row_tile + 1;
     rows0 = ((long long)bi * a.n_q_head + hq) * P + (long long)row_tile * kTM;
   } else {
-    hk = blockIdx.y;
-    row_tile = blockIdx.x;               // key tile 0 sees every query tile: longest first
+    hk = blockIdx.x;
+    row_tile = blockIdx.z;               // key tile 0 sees every query tile: longest first
     n_stream = g * (n_tile - row_tile);
     rows0 = ((long long)bi * a.n_kv_head + hk) * P + (long long)row_tile * kTM;
   }
@@ -317,16 +319,16 @@ static cudaError_t launch_tc_t(const ScoreArgs& a, int* status, cudaStream_t s) 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  k1<<<dim3(n_tile, a.n_q_head, a.batch), kPrefillThreads, smem, s>>>(tm_q, tm_k, a, scale_log2, status);
+  k1<<<dim3(a.n_q_head, a.batch, n_tile), kPrefillThreads, smem, s>>>(tm_q, tm_k, a, scale_log2, status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k2<<<dim3(n_tile, a.n_kv_head, a.batch), kPrefillThreads, smem, s>>>(tm_k, tm_q, a, scale_log2, status);
+  k2<<<dim3(a.n_kv_head, a.batch, n_tile), kPrefillThreads, smem, s>>>(tm_k, tm_q, a, scale_log2, status);
   return cudaGetLastError();
 }
 
 // Returns cudaErrorNotSupported when the shape or the driver cannot serve the tensor-core path.
 cudaError_t launch_prefill_scores_tc(const ScoreArgs& a, int* status, cudaStream_t s) {
-  if (a.n_q_head > 65535 || a.batch > 65535) return cudaErrorNotSupported;
+  if (a.n_q_head > 65535 || a.batch > 65535 || (a.prompt + kTM - 1) / kTM > 65535) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(a.q) | reinterpret_cast<uintptr_t>(a.k)) & 15u) return cudaErrorNotSupported;
   if (a.head_dim == 64) return launch_tc_t<64, 4>(a, status, s);
   if (a.head_dim == 128) return launch_tc_t<128, 2>(a, status, s);
