@@ -699,7 +699,9 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
     }
   }
   if (n_active > 0) {
-    // all descriptors of the call in one launch
+    // all descriptors of the call in one launch, the longest caches first (their CTAs run longest)
+    std::stable_sort(c->hs.evict_tab, c->hs.evict_tab + n_active,
+                     [](const EvictLayer& x, const EvictLayer& y) { return x.len > y.len; });
     EvictArgs a;
     a.pool = c->pool;
     a.tab = ws_ptr<EvictLayer>(c, c->wl.evict_tab);
