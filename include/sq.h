@@ -192,8 +192,9 @@ int sq_kv_bytes_per_step(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, in
  *   q_prompt [batch, n_q_head, prompt_len, head_dim], k_prompt [batch, n_kv_head, prompt_len,
  *   head_dim] (dtype sq_dtype), acc_out fp32 [batch, n_kv_head, prompt_len]; all device
  *   pointers, 16-byte aligned.  acc_out[b, h, t] = sum over the query heads sharing KV head h
- *   and over rows r >= t of softmax_row_r(Q K^T / sqrt(head_dim))[t], exactly what
- *   sq_prefill_compress computes from q_prompt.
+ *   and over rows r >= t of softmax_row_r(Q K^T / sqrt(head_dim))[t], the quantity
+ *   sq_prefill_compress computes from q_prompt (bf16 inputs take the fp32-pipe kernels here, so the
+ *   two agree to rounding, not bit for bit).
  * Limits and rules:
  *   - batch * n_q_head * prompt_len <= SQ_STATIC_SCORE_MAX_ROWS (the array holds one float
  *     per query row: 4 MiB, resident on every GPU that loads the library until the process
