@@ -122,7 +122,10 @@ def test_prefill_compress_keeps_what_cseq_keeps(policy, dtype, head_dim, budgets
 def test_h2o_prompt_scores_match_oracle():
     for dtype, d, g, P in [(torch.float32, 64, 1, 150), (torch.bfloat16, 128, 4, 150), (torch.bfloat16, 64, 3, 150),
                            (torch.bfloat16, 128, 2, 700), (torch.bfloat16, 64, 5, 513), (torch.bfloat16, 128, 1, 128),
-                           (torch.float32, 128, 2, 200)]:
+                           (torch.float32, 128, 2, 200),
+                           # prompts that leave the second 64-column half of a score tile empty, one column
+                           # wide, or ragged on the last tile (each half is drained by its own warps)
+                           (torch.bfloat16, 128, 2, 40), (torch.bfloat16, 64, 2, 65), (torch.bfloat16, 128, 1, 193)]:
         w = small("score", 16, policy=synth.H2O, dtype=dtype, head_dim=d, n_q_head=2 * g, n_kv_head=2,
                   prompt=P, n_layer=1, heavy_mode="uniform4")
         ctx = H.make_ctx(w, b_init=w.prompt)
