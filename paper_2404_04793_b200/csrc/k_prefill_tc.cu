@@ -16,6 +16,8 @@
 // completion through tcgen05.commit -> mbarrier; warps 2-5 drain the accumulators with
 // tcgen05.ld.  Two accumulator buffers let the next tile's MMA run under this tile's exponentials.
 // Every mbarrier wait is bounded: on expiry the CTA raises a status bit and winds down.
+#include <type_traits>
+
 #include "sq_internal.h"
 #include "sq_tc.cuh"
 
@@ -195,47 +197,54 @@ __global__ void __launch_bounds__(kPrefillThreads, 2)
       if (ok) ok = mbar_wait(bar_sfull(buf), (i >> 1) & 1, abort_flag);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const bool diag = (qt == row_tile);
+      // The tile on the diagonal masks half of its elements; every other tile masks none.  The two
+      // cases are separate instantiations of the drain loop, so that tiles off the diagonal (all
+      // but one per row of tiles) carry no compare / select per element.
+      auto drain_tile = [&](auto diag_c) {
+        constexpr bool DIAG = decltype(diag_c)::value;
 #pragma unroll 1
-      for (int c = 2 * half; c < 2 * half + 2; ++c) {
-        float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTM + c * 32, v);
-        if (SWEEP == 1) {
-          if (diag) {
+        for (int c = 2 * half; c < 2 * half + 2; ++c) {
+          float v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTM + c * 32, v);
+          if (SWEEP == 1) {
+            if (DIAG) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c * 32 + j > row) v[j] = -INFINITY;  // key after the query
-          }
-          float mx = v[0];
+              for (int j = 0; j < 32; ++j)
+                if (c * 32 + j > row) v[j] = -INFINITY;  // key after the query
+            }
+            float mx = v[0];
 #pragma unroll
-          for (int j = 1; j < 32; ++j) mx = fmaxf(mx, v[j]);
-          const float m_new = fmaxf(m, mx * scale_log2);
-          if (m_new > -INFINITY) {
-            float sum = 0.f;
+            for (int j = 1; j < 32; ++j) mx = fmaxf(mx, v[j]);
+            const float m_new = fmaxf(m, mx * scale_log2);
+            if (m_new > -INFINITY) {
+              float sum = 0.f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) sum += ex2(fmaf(v[j], scale_log2, -m_new));
-            l = l * ex2(m - m_new) + sum;
-            m = m_new;
-          }
-        } else {
-          const float4* ls = reinterpret_cast<const float4*>(lse_s + buf * kTM + c * 32);
+              for (int j = 0; j < 32; ++j) sum += ex2(fmaf(v[j], scale_log2, -m_new));
+              l = l * ex2(m - m_new) + sum;
+              m = m_new;
+            }
+          } else {
+            const float4* ls = reinterpret_cast<const float4*>(lse_s + buf * kTM + c * 32);
 #pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4) {
-            const float4 lv = ls[j4];
-            const float e0 = ex2(fmaf(v[4 * j4 + 0], scale_log2, -lv.x));
-            const float e1 = ex2(fmaf(v[4 * j4 + 1], scale_log2, -lv.y));
-            const float e2 = ex2(fmaf(v[4 * j4 + 2], scale_log2, -lv.z));
-            const float e3 = ex2(fmaf(v[4 * j4 + 3], scale_log2, -lv.w));
-            if (diag) {
-              const int q0 = c * 32 + 4 * j4;  // query before the key: no attention
-              colsum += (q0 + 0 >= row ? e0 : 0.f) + (q0 + 1 >= row ? e1 : 0.f) + (q0 + 2 >= row ? e2 : 0.f) +
-                        (q0 + 3 >= row ? e3 : 0.f);
-            } else {
-              colsum += (e0 + e1) + (e2 + e3);
+            for (int j4 = 0; j4 < 8; ++j4) {
+              const float4 lv = ls[j4];
+              const float e0 = ex2(fmaf(v[4 * j4 + 0], scale_log2, -lv.x));
+              const float e1 = ex2(fmaf(v[4 * j4 + 1], scale_log2, -lv.y));
+              const float e2 = ex2(fmaf(v[4 * j4 + 2], scale_log2, -lv.z));
+              const float e3 = ex2(fmaf(v[4 * j4 + 3], scale_log2, -lv.w));
+              if (DIAG) {
+                const int q0 = c * 32 + 4 * j4;  // query before the key: no attention
+                colsum += (q0 + 0 >= row ? e0 : 0.f) + (q0 + 1 >= row ? e1 : 0.f) + (q0 + 2 >= row ? e2 : 0.f) +
+                          (q0 + 3 >= row ? e3 : 0.f);
+              } else {
+                colsum += (e0 + e1) + (e2 + e3);
+              }
             }
           }
         }
-      }
+      };
+      if (qt == row_tile) drain_tile(std::true_type{});
+      else drain_tile(std::false_type{});
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(bar_sfree(buf));
     }
