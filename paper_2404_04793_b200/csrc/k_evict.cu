@@ -41,6 +41,24 @@ __device__ __forceinline__ void cp_async_wait_all_but(int n) {
     default: asm volatile("cp.async.wait_group 5;"); break;
   }
 }
+
+// H2O: among the first b slots, the token outside the recent window (position <= last_old) that
+// goes first: smallest score, on equal scores the highest position.  -1 if there is none.
+__device__ __forceinline__ int h2o_next_victim(SelScratch& sc, const int* pos, const float* acc, int b, int last_old) {
+  unsigned long long best = ~0ull;
+  int slot = -1;
+  for (int i = threadIdx.x; i < b; i += kSelThreads) {
+    const int p = pos[i];
+    if (p <= last_old) {
+      const unsigned long long r = victim_rank(acc[i], p);
+      if (r < best) {
+        best = r;
+        slot = i;
+      }
+    }
+  }
+  return block_argmin(sc, best, slot);
+}
 }  // namespace
 
 // Dynamic shared memory: kStages chunks of rows, then per stage the chunk's positions and
@@ -64,7 +82,15 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
   int* pos = reinterpret_cast<int*>(a.pool + lo.pos_off) + (size_t)unit * cap;
   float* acc = reinterpret_cast<float*>(a.pool + lo.acc_off) + (size_t)unit * cap;
   const bool h2o = (a.policy == SQ_POLICY_H2O);
-  if (n <= b) return;
+  if (n <= b) {
+    // nothing to drop.  A cache that the new budget makes exactly full still needs the slot its
+    // next append replaces (H2O): no earlier kernel has chosen one while it was below budget.
+    if (h2o && n == b) {
+      const int slot = h2o_next_victim(sc, pos, acc, b, n_tok - ln.b_recent);
+      if (tid == 0) reinterpret_cast<int*>(a.pool + lo.victim_off)[unit] = slot;
+    }
+    return;
+  }
 
   // --- which slots stay ---
   int recent_from;  // positions >= recent_from are kept as "recent"
@@ -198,20 +224,7 @@ __global__ void __launch_bounds__(kSelThreads) evict_kernel(EvictArgs a) {
 
   // --- H2O: the slot the next append replaces ---
   if (h2o) {
-    const int vthr = n_tok - ln.b_recent;
-    unsigned long long best = ~0ull;
-    int slot = -1;
-    for (int i = tid; i < b; i += kSelThreads) {
-      int p = pos[i];
-      if (p <= vthr) {
-        unsigned long long r = victim_rank(acc[i], p);
-        if (r < best) {
-          best = r;
-          slot = i;
-        }
-      }
-    }
-    slot = block_argmin(sc, best, slot);
+    const int slot = h2o_next_victim(sc, pos, acc, b, n_tok - ln.b_recent);
     if (tid == 0) reinterpret_cast<int*>(a.pool + lo.victim_off)[unit] = slot;
   }
 }

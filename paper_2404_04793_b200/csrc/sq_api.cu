@@ -686,7 +686,9 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
           nw.ring_origin = x0 - h;
         }
       }
-      if (len > nb) {
+      // a cache the new budget makes exactly full has nothing to drop, but under H2O the kernel
+      // still has to choose the slot its next append replaces
+      if (len > nb || (len == nb && cfg.policy == SQ_POLICY_H2O)) {
         EvictLayer& ev = c->hs.evict_tab[n_active++];
         ev.ld_old = old;
         ev.ld_new = nw;

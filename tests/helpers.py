@@ -74,16 +74,18 @@ def all_units(w):
     return [(l, s, h) for l in range(w.n_layer) for s in range(w.batch) for h in range(w.n_kv_head)]
 
 
-def sample_units(w, n, seed=0):
+def sample_units(w, n, seed=0, every_layer=True):
+    """Seeded sample of (layer, sequence, KV head) units: always the first and the last unit and,
+    with every_layer, every layer of one sequence and head (so at least n_layer + 2 units)."""
     units = all_units(w)
     if len(units) <= n:
         return units
     rng = np.random.default_rng(seed)
     pick = {0, len(units) - 1}
-    # every layer of one sequence / head
     s0, h0 = int(rng.integers(w.batch)), int(rng.integers(w.n_kv_head))
-    for l in range(w.n_layer):
-        pick.add((l * w.batch + s0) * w.n_kv_head + h0)
+    if every_layer:
+        for l in range(w.n_layer):
+            pick.add((l * w.batch + s0) * w.n_kv_head + h0)
     while len(pick) < n:
         pick.add(int(rng.integers(len(units))))
     return [units[i] for i in sorted(pick)]

@@ -1,5 +1,8 @@
-"""Multi-rank plumbing on CPU (gloo, world_size 2): the barrier / sum / max helpers that
-bench.py uses to turn per-rank device times into whole-job throughput."""
+"""Multi-rank plumbing on CPU (gloo, world_size 2): the launcher that `bench.py --gpus N` uses to
+start its ranks, and the barrier / sum / max helpers that turn per-rank device times into
+whole-job throughput."""
+import json
+import sys
 import os
 import socket
 
@@ -51,3 +54,43 @@ def test_single_process_helpers_need_no_group():
     from paper_2404_04793_b200 import dist_util
     assert dist_util.max_over_ranks(3.5) == 3.5
     assert dist_util.aggregate_throughput(100, 20.0) == (5000.0, 20.0)
+
+
+STUB = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_stub_job.py")
+
+
+def test_launcher_starts_two_ranks_and_rank0_reports():
+    """The launcher bench.py calls for --gpus 2, driving a stub job over gloo: both ranks run,
+    meet in the barrier and the reductions, and rank 0 prints the whole-job line."""
+    from paper_2404_04793_b200 import dist_util
+    rc, text = dist_util.spawn_ranks(2, [sys.executable, STUB], capture_rank0=True, timeout=240)
+    assert rc == 0, text
+    line = json.loads(text.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2
+    assert line["ms_per_step"] == 50.0                       # the slowest rank sets the time
+    assert line["value"] == pytest.approx(2048 / 0.050)      # tokens of both ranks
+
+
+def test_launcher_reports_a_failed_rank_and_stops_the_rest():
+    from paper_2404_04793_b200 import dist_util
+    rc = dist_util.spawn_ranks(2, [sys.executable, STUB, "--fail-rank", "1"], timeout=240,
+                               extra_env={"TORCH_GLOO_TIMEOUT": "20"})
+    assert rc != 0
+
+
+def test_bench_spawns_ranks_itself_when_asked_for_several_gpus(monkeypatch):
+    """`python bench.py --gpus 2` without RANK in the environment must go through the launcher
+    with its own command line; under a launcher (RANK set) it must not spawn again."""
+    import importlib
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    bench = importlib.import_module("bench")
+    calls = []
+    from paper_2404_04793_b200 import dist_util
+    monkeypatch.setattr(dist_util, "spawn_ranks", lambda n, argv, **kw: calls.append((n, list(argv))) or 0)
+    monkeypatch.delenv("RANK", raising=False)
+    assert bench.maybe_spawn(["--gpus", "2", "--steps", "1"], 2) == 0
+    assert calls and calls[0][0] == 2 and calls[0][1][-4:] == ["--gpus", "2", "--steps", "1"]
+    monkeypatch.setenv("RANK", "0")
+    assert bench.maybe_spawn(["--gpus", "2"], 2) is None and len(calls) == 1
+    assert bench.maybe_spawn(["--gpus", "1"], 1) is None

@@ -359,6 +359,49 @@ def test_evict_in_place_then_keep_decoding(policy):
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("dtype,head_dim,hq,hkv", [(torch.float32, 64, 4, 2), (torch.bfloat16, 128, 8, 2),
+                                                  (torch.bfloat16, 64, 71, 1)])
+def test_evict_of_a_growing_h2o_cache_to_exactly_its_length(dtype, head_dim, hq, hkv):
+    """A cache still below its budget (prompt 20, budget 40, 10 steps -> 30 tokens) is lowered to
+    a budget equal to its length: nothing is dropped, but the very next step is over budget, so
+    the slot that step reuses has to be chosen by the eviction call itself."""
+    w = small("evict_eq", 27, policy=synth.H2O, dtype=dtype, head_dim=head_dim, n_q_head=hq, n_kv_head=hkv,
+              prompt=20, heavy_mode="uniform4", steps=13)
+    budgets = [40, 40, 25]
+    ctx = H.make_ctx(w, b_init=max(budgets))
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets(budgets)
+    prompt_cpu = H.prefill_all(ctx, w, DEV)
+    units = H.all_units(w)
+    oracles = {u: H.oracle_unit(w, budgets, prompt_cpu, *u) for u in units}
+    g = w.group
+
+    def step(t):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+        qc, kc, vc, oc = q.cpu(), kn.cpu(), vn.cpu(), out.cpu()
+        for (l, s, h) in units:
+            u = oracles[(l, s, h)]
+            want = u.decode_step(H.f64(qc[l, s, h * g:(h + 1) * g]), H.f64(kc[l, s, h]), H.f64(vc[l, s, h]))
+            assert np.max(np.abs(H.f64(oc[l, s, h * g:(h + 1) * g]) - want)) <= H.TOL_OUT[w.dtype], (t, l, s, h)
+            pos, acc = ctx.get_kept(l, s, h)
+            assert pos == u.kept_positions(), (t, l, s, h)
+            assert np.allclose(acc, u.acc, rtol=H.RTOL_ACC[w.dtype], atol=1e-6), (t, l, s, h)
+
+    for t in range(10):
+        step(t)
+    new_budgets = [30, 35, 25]          # exactly the length / still above it / unchanged (already full)
+    ctx.evict(0, w.n_layer, new_budgets)
+    for (l, s, h) in units:
+        oracles[(l, s, h)].b = new_budgets[l]
+        oracles[(l, s, h)]._compress()
+        assert ctx.get_kept(l, s, h)[0] == oracles[(l, s, h)].kept_positions()
+    for t in range(10, w.steps):
+        step(t)
+    assert ctx.status() == 0
+
+
 # ----------------------------------------------------------------- error paths
 def test_call_order_and_argument_errors():
     w = small("err", 26)

@@ -1,6 +1,8 @@
 """Seeded random sweep over shapes, policies, budgets and call forms: the CUDA library against
 the oracle on sampled units, including an explicit eviction to random tighter budgets.
 Kept sets, cached rows and budgets must be identical; outputs within the max-abs tolerance.
+A free-running H2O kept set may differ from the oracle's only in one token whose fp64 score ties
+the other's to within the accuracy of the fp32 scores; such steps are verified, counted and printed.
 Where the exact output exceeds 1 in magnitude the bf16 formats themselves limit the agreement
 (output rounding 2^-9..2^-8 relative, weights entering P.V rounded 2^-9 relative), so the bound
 there is 2^-7 of the exact value; below that it is the plain 1e-2 (bf16) / 1e-5 (fp32)."""
@@ -10,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import sq_oracle as O
 from paper_2404_04793_b200 import synth
 from tests import helpers as H
 
@@ -26,9 +29,33 @@ def _check_out(got, want, dtype, where):
     assert np.all(np.abs(got - want) <= bound), where
 
 
+def _near_tie(kept_oracle, kept_gpu, score, b, hn, hd, dtype, where):
+    """The one allowed difference between a free-running H2O kept set and the oracle's: exactly
+    one token differs, both lie outside the recent window, and their fp64 scores (`score`: position
+    -> score of every token that competed) agree to within the accuracy the fp32 scores are held
+    to.  Returns the margin."""
+    only_o, only_g = set(kept_oracle) - set(kept_gpu), set(kept_gpu) - set(kept_oracle)
+    assert len(only_o) == 1 and len(only_g) == 1, (where, only_o, only_g)
+    x, y = only_o.pop(), only_g.pop()
+    recent = sorted(score)[len(score) - (b - (b * hn) // hd):]
+    assert x not in recent and y not in recent, (where, x, y)
+    margin = abs(score[x] - score[y])
+    assert margin <= 2 * H.RTOL_ACC[dtype] * max(abs(score[x]), abs(score[y])) + 1e-6, (where, x, y, score[x], score[y])
+    return margin
+
+
+def _adopt_gpu_state(ctx, u, key):
+    """Carry on from the library's state, so that later steps and the eviction are still checked."""
+    pos, acc = ctx.get_kept(*key)
+    kk, vv = ctx.get_kv(*key)
+    u.pos, u.acc = list(pos), [float(a) for a in acc]
+    u.K, u.V = list(H.f64(kk)), list(H.f64(vv))
+
+
 @pytest.mark.parametrize("seed", [11, 12, 13])
 def test_random_configurations(seed):
     rng = random.Random(seed)
+    near_ties = []
     for case in range(24):
         dtype, d, hq, hkv = rng.choice(SHAPES)
         policy = rng.choice([synth.SLIDING_WINDOW, synth.STREAMING_LLM, synth.H2O])
@@ -58,7 +85,17 @@ def test_random_configurations(seed):
         oracles = {(l, s, h): H.oracle_unit(w, budgets[s] if per_seq else budgets, prompt_cpu, l, s, h)
                    for (l, s, h) in units}
         g = w.group
-        diverged = False
+        for (l, s, h) in units:          # the prompt's own compression
+            u = oracles[(l, s, h)]
+            got_pos = ctx.get_kept(l, s, h)[0]
+            if got_pos != u.kept_positions():
+                assert policy == synth.H2O, (tag, "prefill", l, s, h)
+                qp, kp, _ = prompt_cpu[l]
+                full = O.prefill_scores(H.f64(qp[s, h * g:(h + 1) * g]), H.f64(kp[s, h]))
+                margin = _near_tie(u.kept_positions(), got_pos, dict(enumerate(full)), u.b, hn, hd, dtype,
+                                   (tag, "prefill", l, s, h))
+                near_ties.append((seed, case, -1, l, s, h, margin))
+                _adopt_gpu_state(ctx, u, (l, s, h))
         for t in range(steps):
             q, kn, vn = synth.decode_qkv(w, t, DEV)
             out = torch.empty_like(q)
@@ -70,24 +107,32 @@ def test_random_configurations(seed):
             qc, kc, vc, oc = q.cpu(), kn.cpu(), vn.cpu(), out.cpu()
             for (l, s, h) in units:
                 u = oracles[(l, s, h)]
+                before = (list(u.pos), list(u.acc))
                 want = u.decode_step(H.f64(qc[l, s, h * g:(h + 1) * g]), H.f64(kc[l, s, h]), H.f64(vc[l, s, h]))
-                _check_out(H.f64(oc[l, s, h * g:(h + 1) * g]), want, dtype, (tag, t, l, s, h))
-                if ctx.get_kept(l, s, h)[0] != u.kept_positions():
-                    # only a free-running H2O trajectory may leave the oracle's (near-tied scores)
+                got_pos, got_acc = ctx.get_kept(l, s, h)
+                if got_pos != u.kept_positions():
+                    # Only a free-running H2O trajectory may leave the oracle's, and only where the
+                    # oracle itself could not tell the two tokens apart: exactly one token differs,
+                    # both lie outside the recent window, and their fp64 scores before this step's
+                    # compression agree to within the accuracy the fp32 scores are held to.
                     assert policy == synth.H2O, (tag, t, l, s, h)
-                    diverged = True
-            if diverged:
-                break
-        if not diverged:
-            newb = [[rng.randint(lo, b) for b in r] for r in budgets] if per_seq else [rng.randint(lo, b) for b in budgets]
-            ctx.evict(0, L, newb)
-            for (l, s, h) in units:
-                u = oracles[(l, s, h)]
-                u.b = newb[s][l] if per_seq else newb[l]
-                u._compress()
-                assert ctx.get_kept(l, s, h)[0] == u.kept_positions(), (tag, "evict", l, s, h)
-                if u.K:
-                    k, v = ctx.get_kv(l, s, h)
-                    assert np.array_equal(H.f64(k), np.stack(u.K)) and np.array_equal(H.f64(v), np.stack(u.V)), (tag, l, s, h)
+                    score = dict(zip(before[0], before[1]))
+                    score[w.prompt + t] = 0.0
+                    margin = _near_tie(u.kept_positions(), got_pos, score, u.b, hn, hd, dtype, (tag, t, l, s, h))
+                    near_ties.append((seed, case, t, l, s, h, margin))
+                    _adopt_gpu_state(ctx, u, (l, s, h))
+                else:
+                    _check_out(H.f64(oc[l, s, h * g:(h + 1) * g]), want, dtype, (tag, t, l, s, h))
+        newb = [[rng.randint(lo, b) for b in r] for r in budgets] if per_seq else [rng.randint(lo, b) for b in budgets]
+        ctx.evict(0, L, newb)
+        for (l, s, h) in units:
+            u = oracles[(l, s, h)]
+            u.b = newb[s][l] if per_seq else newb[l]
+            u._compress()
+            assert ctx.get_kept(l, s, h)[0] == u.kept_positions(), (tag, "evict", l, s, h)
+            if u.K:
+                k, v = ctx.get_kv(l, s, h)
+                assert np.array_equal(H.f64(k), np.stack(u.K)) and np.array_equal(H.f64(v), np.stack(u.V)), (tag, l, s, h)
         assert ctx.status() == 0, tag
         ctx.close()
+    print(f"seed {seed}: {len(near_ties)} free-running H2O near-tie divergences {near_ties}")

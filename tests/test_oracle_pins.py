@@ -393,12 +393,25 @@ def test_decode_degenerate_cases():
     vn = rng.standard_normal(d)
     out = u.decode_step(rng.standard_normal((1, d)), kk, vn)
     assert np.allclose(out[0], np.vstack([Vp, vn]).mean(axis=0), atol=1e-13)
-    # one query head per KV head (MHA) is the g = 1 case of the grouped form
-    u1 = O.UnitCache(O.H2O, b=6); u2 = O.UnitCache(O.H2O, b=6)
-    Kp = rng.standard_normal((9, d)); Vp = rng.standard_normal((9, d)); Qp = rng.standard_normal((2, 9, d))
-    u1.prefill(Kp, Vp, Qp[:1]); u2.prefill(Kp, Vp, Qp[:1])
-    q = rng.standard_normal((1, d)); kn = rng.standard_normal(d)
-    assert np.array_equal(u1.decode_step(q, kn, vn), u2.decode_step(q.copy(), kn, vn))
+    # one query head per KV head (MHA) is the g = 1 case of the grouped form: two heads run as
+    # two separate g = 1 units must give what plain multi-head attention gives, written here as
+    # its own loop (full cache, so nothing is evicted) with scipy's softmax
+    from scipy.special import softmax
+    P, T, H_ = 9, 3, 2
+    Kp = rng.standard_normal((H_, P, d)); Vp = rng.standard_normal((H_, P, d)); Qp = rng.standard_normal((H_, P, d))
+    units = [O.UnitCache(O.H2O, b=P + T) for _ in range(H_)]
+    for h in range(H_):
+        units[h].prefill(Kp[h], Vp[h], Qp[h:h + 1])
+    Kall = [list(Kp[h]) for h in range(H_)]
+    Vall = [list(Vp[h]) for h in range(H_)]
+    for t in range(T):
+        q = rng.standard_normal((H_, d)); kn = rng.standard_normal((H_, d)); vn2 = rng.standard_normal((H_, d))
+        for h in range(H_):
+            got = units[h].decode_step(q[h:h + 1], kn[h], vn2[h])
+            Kall[h].append(kn[h]); Vall[h].append(vn2[h])
+            w_ = softmax(np.array([np.dot(q[h], kr) for kr in Kall[h]]) / np.sqrt(d))
+            want = sum(w_[i] * Vall[h][i] for i in range(len(w_)))
+            assert got.shape == (1, d) and np.allclose(got[0], want, atol=1e-13)
 
 
 def test_h2o_trajectory_matches_step_by_step_definition():
