@@ -4,19 +4,27 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 A step is one whole pass of the path over one synthetic batch: layer importance for every
-layer, budget allocation, prefill compression of every layer, then all decode steps (one
-fused launch per decode step over all layers).  The metric is generated tokens per second
-(batch * decode steps / pass time).  With N > 1 every rank runs its own independent batch
-(no data-path collective); the value is the sum over ranks / the slowest rank's time.
+layer, budget allocation, prefill compression of every layer, then all decode steps, each
+decode step issued as one launch per layer (what a model that computes a layer's query from the
+previous layer's output has to issue), replayed from a CUDA graph.  The metric is generated
+tokens per second (batch * decode steps / pass time).  The default workload is the largest cell
+of the Falcon-7B-shaped sweep (batch 224, prompt 16384, budget 50 %, Sliding Window: 15 GB of
+K/V read per decode step).  Beside the headline the line carries the same decode steps as one
+fused launch over all layers (an upper bound no model can issue), decode-step records of the
+other paper-shaped configurations, the whole pass of the Llama-2-7B-shaped configuration, the
+pass fed from host memory, and the CPU oracle's timing.
+
+With --gpus N > 1 and no RANK in the environment the script starts N ranks itself (one per
+GPU); every rank runs its own independent batch (no data-path collective) and the value is the
+sum of the ranks' tokens over the slowest rank's time.
 
 --impl reference times the CPU oracle (oracle/), as it stands, on the host cores on a bounded
-sample of the same workload and extrapolates to the whole job.
+sample of the same workload per step and extrapolates to the whole job.
 """
 from __future__ import annotations
 
 import argparse
 import json
-import math
 import os
 import statistics
 import subprocess
@@ -28,22 +36,43 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 import numpy as np
-import torch
 
-from paper_2404_04793_b200 import dist_util, synth
+# torch and the package are imported inside the functions that need them: the worker processes
+# of the all-cores oracle timing import this file and need neither.
 
 METRIC = "decode tokens/sec at 1 B200 and fused attn+evict HBM GB/s as % of roofline"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram bytes (read+write) per decode launch of the default workload, from the ncu capture
-# summarised in profiles/decode_attn_llama2_7b_sw_b2.md (batch-2 capture scaled by 4 to batch 8).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama2_7b_sw_bf16": 1.7373e9}
+DEFAULT_WORKLOAD = "falcon_7b_max"
+# DRAM bytes (read + write) per byte of K/V a decode launch has to read, from ncu captures of each
+# decode kernel on a small case (traffic grows in proportion to the units processed, each unit's
+# K/V being read once); None once a kernel has changed since its counters were taken.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"decode_attn_kernel": 1.008, "decode_attn_tc_kernel": None,
+                                    "decode_attn_mma_kernel": None}
 
 
 def workload_by_name(name):
+    from paper_2404_04793_b200 import synth
     if name not in synth.WORKLOADS:
         raise SystemExit(f"unknown workload {name}; choose from {sorted(synth.WORKLOADS)}")
     return synth.WORKLOADS[name]()
+
+
+def config_of(w, world):
+    """The workload as the JSON line names it (both arms print the same keys)."""
+    from paper_2404_04793_b200 import synth
+    return {"workload": w.name, "n_layer": w.n_layer, "n_q_head": w.n_q_head, "n_kv_head": w.n_kv_head,
+            "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch, "prompt": w.prompt,
+            "decode_steps": w.steps, "policy": synth.POLICY_NAMES[w.policy], "b_init": w.b_init, "p": w.p,
+            "parallelism": f"dp{world} (independent batches)"}
+
+
+def maybe_spawn(argv, gpus):
+    """`--gpus N` outside a launcher: start the N ranks and return their exit code; else None."""
+    if gpus <= 1 or "RANK" in os.environ:
+        return None
+    from paper_2404_04793_b200 import dist_util
+    return dist_util.spawn_ranks(gpus, [sys.executable, os.path.abspath(__file__), *argv])
 
 
 # ------------------------------------------------------------------ clocks
@@ -53,6 +82,7 @@ class ClockSampler:
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, device_index):
+        import torch
         self.uuid = str(torch.cuda.get_device_properties(device_index).uuid)
         self.proc = None
         self.path = os.path.join("/tmp", f"sq_clocks_{os.getpid()}.csv")
@@ -111,72 +141,167 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------ CPU oracle leg
-def oracle_sample(w, n_units, n_imp_tokens, seed, device):
-    """Times the oracle on a bounded sample of the workload and extrapolates linearly to the
-    whole job (units of a layer cost the same; importance cost is per token).
-    Returns (tokens_per_s, seconds_spent, description)."""
+def _one_thread():
     from threadpoolctl import threadpool_limits
-    with threadpool_limits(limits=1):
-        return _oracle_sample(w, n_units, n_imp_tokens, seed, device)
+    return threadpool_limits(limits=1)
 
 
-def _oracle_sample(w, n_units, n_imp_tokens, seed, device):
+def oracle_unit_task(task):
+    """One (layer, sequence, KV head) unit through the oracle: prompt, then every decode step.
+    Returns the seconds it took.  Runs in this process or in a worker of the all-cores pool."""
     from oracle import sq_oracle as O
+    with _one_thread():
+        t0 = time.perf_counter()
+        u = O.UnitCache(task["policy"], task["budget"], task["n_sink"], task["heavy_num"], task["heavy_den"])
+        u.prefill(task["k"], task["v"], task["q"])
+        for (q, kn, vn) in task["steps"]:
+            u.decode_step(q, kn, vn)
+        return time.perf_counter() - t0
+
+
+def oracle_importance_task(task):
+    from oracle import sq_oracle as O
+    with _one_thread():
+        t0 = time.perf_counter()
+        c = O.layer_importance(task["a"], task["b"])
+        return time.perf_counter() - t0, c
+
+
+def oracle_tasks(w, n_units, n_imp_tokens, seed, device):
+    """Draws a bounded sample of the workload for the oracle: importance chunks (a few layers,
+    n_imp_tokens tokens in all) and n_units (layer, sequence, KV head) units with all their decode
+    steps.  Returns (importance tasks, unit tasks, budgets)."""
+    import torch
+    from oracle import sq_oracle as O
+    from paper_2404_04793_b200 import synth
     rng = np.random.default_rng(seed)
     f64 = lambda t: t.detach().to("cpu").to(torch.float64).numpy()
-    t_start = time.perf_counter()
-    # importance: first n_imp_tokens tokens of every 8th layer (cost per token is the same)
     layers_imp = list(range(0, w.n_layer, max(1, w.n_layer // 4)))[:4]
     per_layer = max(1, n_imp_tokens // len(layers_imp))
-    cos = np.array(synth.cos_targets(w.n_layer), dtype=np.float64)
-    t_imp = 0.0
-    n_imp = 0
+    imp = []
     for l in layers_imp:
-        nb = max(1, min(w.batch, per_layer // w.prompt))
-        a, b = synth.hidden_pair(w, l, device, batch=nb, n_tok=min(per_layer, w.prompt))
-        a, b = f64(a), f64(b)
-        t0 = time.perf_counter()
-        cos[l] = O.layer_importance(a, b)
-        t_imp += time.perf_counter() - t0
-        n_imp += a.shape[0] * a.shape[1] if a.ndim == 3 else a.shape[0]
-    t0 = time.perf_counter()
-    budgets, _ = O.allocate_budgets(cos.astype(np.float32), w.b_init, w.p)
-    t_alloc = time.perf_counter() - t0
-    # decode: sampled (layer, sequence, KV head) units, spread evenly over the layers
-    layers = sorted(set(int(x) for x in np.linspace(0, w.n_layer - 1, min(n_units, w.n_layer)).round()))
+        a, b = synth.hidden_pair(w, l, device, batch=1, n_tok=min(per_layer, w.prompt))
+        imp.append({"layer": l, "a": f64(a[0]), "b": f64(b[0])})
+    # budgets from the generator's target similarities (the sampled layers are re-measured by the oracle)
+    cos = np.array(synth.cos_targets(w.n_layer), dtype=np.float32)
+    budgets, is_g3 = O.allocate_budgets(cos, w.b_init, w.p)
+    # sampled layers: spread evenly within each budget class (the least important group / the rest)
+    classes = [[l for l in range(w.n_layer) if bool(is_g3[l]) == c] for c in (False, True)]
+    classes = [c for c in classes if c]
+    per_class = -(-min(n_units, w.n_layer) // len(classes))
+    layers = set()
+    for members in classes:
+        for i in np.linspace(0, len(members) - 1, min(per_class, len(members))).round():
+            layers.add(members[int(i)])
+    layers = sorted(layers)
     per = max(1, n_units // len(layers))
     g = w.group
-    t_units = {}
-    dec = [synth.decode_qkv(w, t, device) for t in range(w.steps)]
+    units = []
     for l in layers:
         q, k, v = synth.prompt_qkv(w, l, device, need_q=(w.policy == synth.H2O))
-        spent = 0.0
         for _ in range(per):
             s, h = int(rng.integers(w.batch)), int(rng.integers(w.n_kv_head))
-            kk, vv = f64(k[s, h]), f64(v[s, h])
-            qq = None if q is None else f64(q[s, h * g:(h + 1) * g])
-            steps = [(f64(dq[l, s, h * g:(h + 1) * g]), f64(dk[l, s, h]), f64(dv[l, s, h])) for dq, dk, dv in dec]
-            t0 = time.perf_counter()
-            u = O.UnitCache(w.policy, int(budgets[l]), w.n_sink, w.heavy_num, w.heavy_den)
-            u.prefill(kk, vv, qq)
-            for (a1, a2, a3) in steps:
-                u.decode_step(a1, a2, a3)
-            spent += time.perf_counter() - t0
-        t_units[l] = spent / per
-    # extrapolate: layers not sampled take the cost of the nearest sampled layer with the same budget class
+            units.append({"layer": l, "seq": s, "head": h, "policy": w.policy, "budget": int(budgets[l]),
+                          "n_sink": w.n_sink, "heavy_num": w.heavy_num, "heavy_den": w.heavy_den, "k": f64(k[s, h]),
+                          "v": f64(v[s, h]), "q": None if q is None else f64(q[s, h * g:(h + 1) * g]), "steps": []})
+        del q, k, v
+    for t in range(w.steps):
+        dq, dk, dv = synth.decode_qkv(w, t, device)
+        for u in units:
+            l, s, h = u["layer"], u["seq"], u["head"]
+            u["steps"].append((f64(dq[l, s, h * g:(h + 1) * g]), f64(dk[l, s, h]), f64(dv[l, s, h])))
+        del dq, dk, dv
+    return imp, units, budgets
+
+
+def extrapolate(w, budgets, imp_s_per_token, alloc_s, unit_s_by_layer):
+    """Whole-job seconds from the sampled costs: importance per token; a unit costs what the
+    sampled layer with the nearest budget (then the nearest index) costs."""
+    layers = sorted(unit_s_by_layer)
+
     def unit_cost(l):
-        same = [x for x in layers if budgets[x] == budgets[l]] or layers
-        return t_units[min(same, key=lambda x: abs(x - l))]
-    t_job = (t_imp / max(n_imp, 1)) * (w.n_layer * w.batch * w.prompt) + t_alloc \
+        return unit_s_by_layer[min(layers, key=lambda x: (abs(int(budgets[x]) - int(budgets[l])), abs(x - l)))]
+
+    return imp_s_per_token * (w.n_layer * w.batch * w.prompt) + alloc_s \
         + sum(unit_cost(l) * w.batch * w.n_kv_head for l in range(w.n_layer))
-    tok_s = w.batch * w.steps / t_job
-    desc = (f"{len(layers) * per} (layer,seq,kv-head) units over {len(layers)} layers, all {w.steps} decode steps, "
-            f"+ {n_imp} tokens of layer importance + the allocator; extrapolated linearly to "
-            f"{w.n_layer * w.batch * w.n_kv_head} units and {w.n_layer * w.batch * w.prompt} tokens")
-    return tok_s, time.perf_counter() - t_start, desc
+
+
+def oracle_sample(w, n_units, n_imp_tokens, seed, device, pool_cores=0):
+    """Times the oracle on a bounded sample of the workload and extrapolates linearly to the
+    whole job.  One thread in this process; with pool_cores > 1 the same kind of sample, pool_cores
+    times as large, is then also run as a plain parallel-for over that many worker processes.
+    Returns a dict with tokens/s (one core), seconds spent, a description and, if asked for, the
+    all-cores figures."""
+    from oracle import sq_oracle as O
+    t_start = time.perf_counter()
+    n_total = n_units * max(1, pool_cores)
+    imp, units, budgets = oracle_tasks(w, n_total, n_imp_tokens * max(1, pool_cores), seed, device)
+    # ---- one core: the first n_units-worth of the sample (spread over the layers) ----
+    stride = max(1, len(units) // max(1, n_units))
+    mine = units[::stride][:n_units]
+    imp_one = imp if pool_cores <= 1 else [{"layer": t["layer"], "a": t["a"][:max(1, len(t["a"]) // pool_cores)],
+                                            "b": t["b"][:max(1, len(t["b"]) // pool_cores)]} for t in imp]
+    t_imp, n_imp = 0.0, 0
+    for t in imp_one:
+        s, _ = oracle_importance_task(t)
+        t_imp += s
+        n_imp += t["a"].shape[0]
+    with _one_thread():
+        t0 = time.perf_counter()
+        O.allocate_budgets(np.array([0.7] * (w.n_layer // 2) + [0.95] * (w.n_layer - w.n_layer // 2), dtype=np.float32),
+                           w.b_init, w.p)
+        t_alloc = time.perf_counter() - t0
+    by_layer = {}
+    for t in mine:
+        by_layer.setdefault(t["layer"], []).append(oracle_unit_task(t))
+    unit_s = {l: sum(v) / len(v) for l, v in by_layer.items()}
+    t_job = extrapolate(w, budgets, t_imp / max(n_imp, 1), t_alloc, unit_s)
+    total_units = w.n_layer * w.batch * w.n_kv_head
+    out = {"value": w.batch * w.steps / t_job, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": (f"{len(mine)} (layer,seq,kv-head) units over {len(unit_s)} layers, all {w.steps} decode steps, "
+                      f"+ {n_imp} tokens of layer importance + the allocator; extrapolated linearly to "
+                      f"{total_units} units and {w.n_layer * w.batch * w.prompt} tokens"),
+           "job_seconds_extrapolated": t_job}
+    # ---- all cores: a plain parallel-for over independent units (and importance chunks) ----
+    if pool_cores > 1:
+        import multiprocessing as mp
+        ctx = mp.get_context("spawn")          # CUDA may already be initialised in this process: never fork
+        with ctx.Pool(pool_cores) as pool:
+            pool.map(abs, range(pool_cores))   # workers up and imported before the clock starts
+            t0 = time.perf_counter()
+            r_imp = pool.map(oracle_importance_task, [{"layer": t["layer"], "a": c_a, "b": c_b} for t in imp
+                                                      for c_a, c_b in zip(np.array_split(t["a"], pool_cores),
+                                                                          np.array_split(t["b"], pool_cores)) if len(c_a)])
+            wall_imp = time.perf_counter() - t0
+            t0 = time.perf_counter()
+            r_units = pool.map(oracle_unit_task, units, chunksize=1)
+            wall_units = time.perf_counter() - t0
+        n_imp_all = sum(t["a"].shape[0] for t in imp)
+        # wall time per unit of work under the parallel-for, weighted like the one-core figure
+        cpu_by_layer = {}
+        for t, s in zip(units, r_units):
+            cpu_by_layer.setdefault(t["layer"], []).append(s)
+        speedup_units = sum(r_units) / wall_units
+        unit_wall = {l: (sum(v) / len(v)) / speedup_units for l, v in cpu_by_layer.items()}
+        t_job_all = extrapolate(w, budgets, wall_imp / max(n_imp_all, 1), t_alloc, unit_wall)
+        out["all_cores"] = {"value": w.batch * w.steps / t_job_all, "unit": UNIT, "cores": pool_cores,
+                            "sample": f"{len(units)} units and {n_imp_all} importance tokens as a parallel-for over "
+                                      f"{pool_cores} worker processes (one thread each); extrapolated the same way",
+                            "parallel_speedup_on_units": speedup_units}
+    out["seconds"] = time.perf_counter() - t_start
+    return out
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
 
 
 def run_reference(args, w):
+    import torch
+    from paper_2404_04793_b200 import dist_util
     rank, local_rank, world = dist_util.world()
     if rank != 0:
         return
@@ -184,17 +309,17 @@ def run_reference(args, w):
     vals, secs = [], []
     desc = ""
     for i in range(args.warmup + args.steps):
-        v, s, desc = oracle_sample(w, n_units=8, n_imp_tokens=4096, seed=100 + i, device=device)
+        r = oracle_sample(w, n_units=2, n_imp_tokens=2048, seed=100 + i, device=device)
         if i >= args.warmup:
-            vals.append(v); secs.append(s)
+            vals.append(r["value"]); secs.append(r["seconds"])
+        desc = r["sample"]
     value = len(vals) / sum(1.0 / v for v in vals)      # steps / total extrapolated time
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch * w.steps / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "prompt": w.prompt, "decode_steps": w.steps,
-                   "policy": synth.POLICY_NAMES[w.policy], "b_init": w.b_init, "p": w.p},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "config": config_of(w, max(1, args.gpus)),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc + " (per step)"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "sample_seconds_per_step": statistics.mean(secs),
     }
@@ -202,28 +327,171 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------ our arm
+def hbm_peak():
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def decode_kernel_of(w):
+    import torch
+    g = w.group
+    if w.dtype == torch.bfloat16 and w.head_dim == 64 and g > 32:
+        return "decode_attn_tc_kernel"
+    if w.dtype == torch.bfloat16 and g > 1:
+        return "decode_attn_mma_kernel"
+    return "decode_attn_kernel"
+
+
+def algorithmic_bytes_per_step(w, kv_bytes):
+    """Bytes one decode step over all layers has to move: K and V of the kept tokens (kv_bytes,
+    from the library's own count at the current fill level), q and out, the new token's k and v,
+    and for H2O the fp32 score of every kept token read and written."""
+    from paper_2404_04793_b200 import synth
+    e = w.dtype.itemsize
+    d, L, B = w.head_dim, w.n_layer, w.batch
+    small = B * L * (w.n_q_head * d * e * 2 + w.n_kv_head * 2 * d * e)
+    acc = (kv_bytes // (2 * d * e)) * 8 if w.policy == synth.H2O else 0
+    return kv_bytes + small + acc
+
+
+def hidden_seqs_for(w, budget_bytes=40e9):
+    """Distinct sequences of hidden states kept per layer: the most that fit budget_bytes."""
+    per_seq = 2 * w.prompt * w.hidden * w.dtype.itemsize * w.n_layer
+    best = 1
+    for s in range(1, w.batch + 1):
+        if w.batch % s == 0 and s * per_seq <= budget_bytes:
+            best = s
+    return best
+
+
+def time_replays(job, inp, graph, n, ev):
+    """Mean milliseconds of n graph replays, each after a fresh prefill of the cache."""
+    import torch
+    tot = 0.0
+    for _ in range(n):
+        job.prefill(inp)
+        a, b = ev(), ev()
+        a.record()
+        graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        tot += a.elapsed_time(b)
+    return tot / n
+
+
+def decode_record(w, dev, peak, n_steps=8, reps=3, standin_scores=False):
+    """Decode-step timing of one configuration: the cache is filled through the library
+    (importance, allocation, prefill compression; outside the timed region), then n_steps decode
+    steps are replayed from CUDA graphs, as one launch per layer and as one fused launch."""
+    import torch
+    from paper_2404_04793_b200 import engine, synth
+    wr = w.replace(steps=n_steps)
+    inp = engine.ResidentInputs(wr, dev, hidden_seqs=1, standin_scores=standin_scores)
+    job = engine.Job(wr, dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    job.prefill(inp)
+    kv = job.ctx.kv_bytes_per_step(0, wr.n_layer)
+    alg = algorithmic_bytes_per_step(wr, kv)
+    budgets, is_g3 = job.ctx.get_budgets()
+    rec = {"workload": w.name, "policy": synth.POLICY_NAMES[w.policy], "batch": w.batch, "prompt": w.prompt,
+           "b_init": w.b_init, "budgets_min_max": [min(budgets), max(budgets)], "kernel": decode_kernel_of(w),
+           "algorithmic_bytes_per_step": alg, "steps_timed": n_steps * reps,
+           "prompt_scores": "stand-in (scoring pass skipped while filling the cache)" if standin_scores else "computed"}
+    for form, per_layer in (("per_layer", True), ("fused", False)):
+        job.prefill(inp)
+        graph = job.capture_decode(inp, per_layer=per_layer)
+        time_replays(job, inp, graph, 1, ev)
+        ms = time_replays(job, inp, graph, reps, ev) / n_steps
+        gbs = alg / (ms * 1e-3) / 1e9
+        rec[form] = {"ms_per_step": ms, "gbs": gbs, "frac": gbs / peak, "frac_of_nominal_8000": gbs / 8000.0,
+                     "tokens_per_s": w.batch / (ms * 1e-3)}
+        del graph
+    rec["device_status"] = job.ctx.status()
+    job.ctx.close()
+    del job, inp
+    torch.cuda.empty_cache()
+    return rec
+
+
+def whole_pass_record(w, dev, peak, reps=3):
+    """Whole pass (importance, allocation, prefill compression, all decode steps as per-layer
+    launches from a CUDA graph) of a configuration small enough to keep every input resident."""
+    import torch
+    from paper_2404_04793_b200 import engine, synth
+    inp = engine.ResidentInputs(w, dev)
+    job = engine.Job(w, dev, per_layer_decode=True, keep_steps=min(w.steps, 16))
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    job.prefill(inp)
+    graph = job.capture_decode(inp, per_layer=True)
+    job.prefill(inp); graph.replay()
+    torch.cuda.synchronize()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(reps):
+        job.prefill(inp)
+        graph.replay()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    ms_dec = time_replays(job, inp, graph, reps, ev)
+    kv = job.ctx.kv_bytes_per_step(0, w.n_layer)       # after the captured steps: the steady state
+    alg = algorithmic_bytes_per_step(w, kv)
+    gbs = alg * w.steps / (ms_dec * 1e-3) / 1e9
+    rec = {"workload": w.name, "policy": synth.POLICY_NAMES[w.policy], "ms_per_pass": ms,
+           "tokens_per_s": w.batch * w.steps / (ms * 1e-3), "decode_ms_per_step": ms_dec / w.steps,
+           "decode_gbs": gbs, "decode_frac": gbs / peak, "decode_launch": "per_layer (CUDA-graph replay)",
+           "device_status": job.ctx.status()}
+    del graph
+    job.ctx.close()
+    del job, inp
+    torch.cuda.empty_cache()
+    return rec
+
+
+def host_memory_available():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
 def run_ours(args, w):
-    from paper_2404_04793_b200 import engine
+    import torch
+    from paper_2404_04793_b200 import dist_util, engine, synth
     rank, local_rank, world = dist_util.init("nccl")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
+    peak, peak_kind = hbm_peak()
     # every rank owns an independent batch: a different seed family per rank
     wr = w.replace(wid=w.wid + 100 * rank) if world > 1 else w
-    inp = engine.ResidentInputs(wr, dev)
-    job = engine.Job(wr, dev, per_layer_decode=args.per_layer_decode)
+    hs = hidden_seqs_for(wr)
+    inp = engine.ResidentInputs(wr, dev, hidden_seqs=hs)
+    job = engine.Job(wr, dev, per_layer_decode=True, keep_steps=min(wr.steps, 16))
     tokens = wr.batch * wr.steps
-
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    for _ in range(args.warmup):
-        job.run(inp)
+
+    # ---- warm-up: whole passes with plain calls, then the decode steps captured once per form ----
+    job.run(inp)
+    job.prefill(inp)
+    graph_pl = job.capture_decode(inp, per_layer=True)
+    for _ in range(max(0, args.warmup - 1)):
+        job.prefill(inp)
+        graph_pl.replay()
     torch.cuda.synchronize()
     budgets, is_g3 = job.ctx.get_budgets()
+    kv_bytes = job.ctx.kv_bytes_per_step(0, wr.n_layer)     # steady state: every layer at its budget
+    alg_bytes = algorithmic_bytes_per_step(wr, kv_bytes)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        job.run(inp)                      # keeps the GPU busy while the sampler starts up
+        job.prefill(inp); graph_pl.replay()                  # keeps the GPU busy while the sampler starts up
     dist_util.barrier()
     torch.cuda.synchronize()
     t_begin = time.time()
@@ -234,7 +502,7 @@ def run_ours(args, w):
         job.prefill(inp)
         a, b = ev(), ev()
         a.record()
-        job.decode(inp)
+        graph_pl.replay()
         b.record()
         mids.append((a, b))
     e1.record()
@@ -246,40 +514,43 @@ def run_ours(args, w):
     ms_decode = sum(a.elapsed_time(b) for a, b in mids) / args.steps
     status = job.ctx.status()
     value, ms_max = dist_util.aggregate_throughput(tokens, ms_step, dev)
+    del graph_pl
 
-    # ---- per-layer launches (what a model that computes q layer by layer issues), replayed from
-    # a CUDA graph so that the host's launch cost does not enter ----
-    per_layer = None
-    if not args.no_per_layer:
+    # ---- the same decode steps as one fused launch over all layers (upper bound) ----
+    fused = None
+    if not args.no_fused:
         job.prefill(inp)
-        graph = job.capture_decode(inp, per_layer=True)
-        for _ in range(2):
-            job.prefill(inp)
-            graph.replay()
-        torch.cuda.synchronize()
-        n_pl = max(1, min(args.steps, 5))
-        tot = 0.0
-        for _ in range(n_pl):
-            job.prefill(inp)
-            a, b = ev(), ev()
-            a.record()
-            graph.replay()
-            b.record()
-            torch.cuda.synchronize()
-            tot += a.elapsed_time(b)
-        per_layer = {"ms_decode": tot / n_pl, "steps": n_pl}
-        del graph
+        graph_f = job.capture_decode(inp, per_layer=False)
+        time_replays(job, inp, graph_f, 1, ev)
+        ms_f = time_replays(job, inp, graph_f, max(1, min(args.steps, 3)), ev)
+        fused = {"mode": "one launch per decode step over all layers (needs every layer's q at once: an upper "
+                         "bound, not a form a model can issue)",
+                 "decode_tokens_per_s": tokens / (ms_f * 1e-3), "ms_per_token_step": ms_f / wr.steps,
+                 "hbm_gbs": alg_bytes * wr.steps / (ms_f * 1e-3) / 1e9,
+                 "hbm_frac": alg_bytes * wr.steps / (ms_f * 1e-3) / 1e9 / peak}
+        del graph_f
 
-    # ---- end to end: the same pass fed from pinned host memory, outputs copied back ----
+    # ---- end to end: the same pass fed from page-locked host memory, outputs copied back ----
     e2e = None
     if not args.no_e2e:
-        host = engine.ResidentInputs(wr, "cpu", gen_device=dev)
-        out_host = torch.empty(job.out.shape, dtype=job.out.dtype).pin_memory()
+        # what the host holds is sized to its memory (at most 32 GB page-locked): fewer distinct
+        # hidden-state sequences and prompt layers than the device-resident run keeps, if need be.
+        # Layer l then sends the prompt tensors of layer l % n, so the bytes per pass stay the same.
+        avail = host_memory_available() or 64e9
+        host_budget = min(0.3 * avail / max(1, world), 32e9)
+        hs_host = hidden_seqs_for(wr, 0.4 * host_budget)
+        per_layer_prompt = (inp.bytes_per_pass() - 2 * sum(a.numel() * a.element_size() for a, _ in inp.hidden)
+                            - inp.q.numel() * inp.q.element_size()) / wr.n_layer
+        n_pl = wr.n_layer
+        while n_pl > 1 and per_layer_prompt * n_pl > 0.4 * host_budget:
+            n_pl //= 2
+        host = engine.ResidentInputs(wr, "cpu", gen_device=dev, hidden_seqs=hs_host, prompt_layers=n_pl)
+        out_host = torch.empty((2,) + tuple(job.out.shape[1:]), dtype=job.out.dtype, pin_memory=True)
         job.run_from_host(host, out_host)
         torch.cuda.synchronize()
         dist_util.barrier()
         s0, s1 = ev(), ev()
-        n_e2e = max(1, min(args.steps, 3))
+        n_e2e = max(1, min(args.steps, 2))
         s0.record()
         for _ in range(n_e2e):
             job.run_from_host(host, out_host)
@@ -287,62 +558,71 @@ def run_ours(args, w):
         torch.cuda.synchronize()
         dist_util.barrier()
         e2e_val, _ = dist_util.aggregate_throughput(tokens, s0.elapsed_time(s1) / n_e2e, dev)
-        e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": host.bytes(),
-               "d2h_bytes_per_step": out_host.numel() * out_host.element_size(), "steps": n_e2e}
-        del host
+        e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": host.bytes_per_pass(),
+               "d2h_bytes_per_step": wr.steps * out_host[0].numel() * out_host.element_size(), "steps": n_e2e,
+               "host_distinct_prompt_layers": n_pl, "host_hidden_sequences_per_layer": hs_host,
+               "note": "per pass every distinct input tensor crosses PCIe once (a layer's hidden-state chunk is "
+                       "then read hidden_repeat times on the device) and every step's output is copied back"}
+        del host, out_host
 
+    launches = job.kernel_launches_per_pass(inp, per_layer_decode=True) * args.steps
+    hidden_repeat = inp.hidden_repeat
+    job.ctx.close()
+    del job, inp
+    torch.cuda.empty_cache()
     if rank != 0:
         dist_util.shutdown()
         return
 
-    # ---- roofline of the dominant kernel: the fused decode launch ----
-    e = 2 if wr.dtype == torch.bfloat16 else 4
-    d, L, B = wr.head_dim, wr.n_layer, wr.batch
-    kv_tokens = sum(min(wr.prompt + 1, b) for b in budgets)            # per unit, steady state
-    alg_bytes = B * wr.n_kv_head * kv_tokens * 2 * d * e \
-        + B * L * (wr.n_q_head * d * e * 2 + wr.n_kv_head * 2 * d * e) \
-        + (B * wr.n_kv_head * kv_tokens * 8 if wr.policy == synth.H2O else 0)
-    launches_per_step = wr.steps * (wr.n_layer if args.per_layer_decode else 1)
-    sec_per_launch = ms_decode * 1e-3 / launches_per_step
-    bytes_per_launch = alg_bytes / (wr.n_layer if args.per_layer_decode else 1)
+    # ---- roofline of the dominant kernel: the per-layer decode launch ----
+    kernel = decode_kernel_of(wr)
+    n_launch = wr.steps * wr.n_layer
+    sec_per_launch = ms_decode * 1e-3 / n_launch
+    bytes_per_launch = alg_bytes / wr.n_layer
     achieved = bytes_per_launch / sec_per_launch / 1e9
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak = float(json.load(open(peaks_path))["hbm_gbs"]); peak_kind = "measured"
-    else:
-        peak = FALLBACK_HBM_GBS; peak_kind = "fallback"
+    ratio = NCU_TRAFFIC_PER_ALGORITHMIC_BYTE.get(kernel)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if args.per_layer_decode else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wr.name), "peak_kind": peak_kind, "kernel": "decode_attn_kernel",
+                "traffic": None if ratio is None else ratio * bytes_per_launch, "peak_kind": peak_kind,
+                "kernel": kernel, "launch": "one per layer per decode step (average over the layers' budgets)",
                 "algorithmic_bytes_per_launch": bytes_per_launch, "us_per_launch": sec_per_launch * 1e6,
-                "frac_of_nominal_8000": achieved / 8000.0}
+                "frac_of_nominal_8000": achieved / 8000.0,
+                "peak_note": "the measured peak is a copy (read + write); a read-mostly kernel can exceed it slightly"}
+
+    records, whole_pass = None, None
+    if world == 1 and not args.no_records:
+        records = []
+        for wl, standin in ((synth.mistral_7b(), False), (synth.llama2_70b(), False),
+                            (synth.falcon_7b_max(synth.SLIDING_WINDOW), False),
+                            (synth.falcon_7b_max(synth.H2O), True)):
+            if wl.name == wr.name and fused is not None:
+                continue                                      # the headline itself: already in the line
+            records.append(decode_record(wl, dev, peak, standin_scores=standin))
+        if wr.name != synth.llama2_7b().name:
+            whole_pass = whole_pass_record(synth.llama2_7b(), dev, peak)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        v, secs, desc = oracle_sample(wr, n_units=256, n_imp_tokens=65536, seed=7, device=dev)
-        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": secs}
+        cores = min(host_cores(), 32)
+        cpu = oracle_sample(wr, n_units=args.cpu_units, n_imp_tokens=16384, seed=7, device=dev,
+                            pool_cores=cores if cores > 1 else 0)
 
+    cfg = config_of(wr, world)
+    cfg.update({"budgets_min_max": [min(budgets), max(budgets)], "n_g3": int(sum(is_g3)),
+                "decode_launch": "per_layer (one launch per layer per step, CUDA-graph replay)",
+                "hidden_states": f"{hs} distinct sequences per layer, fed {hidden_repeat}x (every token's bytes are read)",
+                "l2": "inputs larger than L2 (K/V read per decode step %.2f GB, %.0f MB per launch)"
+                      % (kv_bytes / 1e9, kv_bytes / wr.n_layer / 1e6)})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if wr.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "n_layer": L, "n_q_head": wr.n_q_head, "n_kv_head": wr.n_kv_head,
-                   "head_dim": d, "batch_per_gpu": B, "prompt": wr.prompt, "decode_steps": wr.steps,
-                   "policy": synth.POLICY_NAMES[wr.policy], "b_init": wr.b_init, "p": wr.p,
-                   "budgets_min_max": [min(budgets), max(budgets)], "n_g3": int(sum(is_g3)),
-                   "decode_launch": "per_layer" if args.per_layer_decode else "all_layers_fused",
-                   "l2": "inputs larger than L2 (KV read per decode step %.2f GB)" % (alg_bytes / 1e9),
-                   "parallelism": f"dp{world} (independent batches)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": job.kernel_launches_per_pass() * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu,
+        "dtype": "bf16" if wr.dtype == torch.bfloat16 else "f32", "data": "synthetic", "config": cfg,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
         "decode_only": {"tokens_per_s": tokens / (ms_decode * 1e-3), "ms_per_token_step": ms_decode / wr.steps,
-                        "prefill_ms": ms_step - ms_decode},
+                        "prefill_ms": ms_step - ms_decode, "hbm_gbs": alg_bytes * wr.steps / (ms_decode * 1e-3) / 1e9,
+                        "hbm_frac": alg_bytes * wr.steps / (ms_decode * 1e-3) / 1e9 / peak},
+        "fused_launch_upper_bound": fused, "decode_records": records, "whole_pass_llama2_7b": whole_pass,
         "device_status": status,
     }
-    if per_layer is not None:
-        pl_s = per_layer["ms_decode"] * 1e-3
-        line["per_layer_launch"] = {"mode": "one launch per layer per step, CUDA-graph replay",
-                                    "decode_tokens_per_s": tokens / pl_s, "us_per_launch": pl_s * 1e6 / (wr.steps * wr.n_layer),
-                                    "hbm_gbs": alg_bytes * wr.steps / pl_s / 1e9, "hbm_frac": alg_bytes * wr.steps / pl_s / 1e9 / peak}
     print(json.dumps(line), flush=True)
     dist_util.shutdown()
 
@@ -350,17 +630,21 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama2_7b")
-    ap.add_argument("--per-layer-decode", action="store_true", help="one decode launch per layer instead of one per step")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps")
+    ap.add_argument("--cpu-units", type=int, default=4, help="units the one-core oracle timing samples")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-per-layer", action="store_true", help="skip the per-layer-launch (CUDA graph) measurement")
+    ap.add_argument("--no-fused", action="store_true", help="skip the fused-launch upper bound")
+    ap.add_argument("--no-records", action="store_true", help="skip the decode-step records of the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    rc = maybe_spawn(sys.argv[1:], args.gpus)
+    if rc is not None:
+        sys.exit(rc)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = workload_by_name(args.workload)
     if args.batch:

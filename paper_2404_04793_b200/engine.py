@@ -31,9 +31,12 @@ class ResidentInputs:
     batch is made of batch / hidden_seqs repeats of them (the importance reduction still reads
     every token's bytes: a layer's chunk is fed that many times).  Default: the whole batch.
     prompt_layers: distinct layers of prompt tensors kept (layer l uses l % prompt_layers);
-    default all."""
+    default all.
+    standin_scores: H2O only: keep stand-in prompt scores (synth.prompt_scores_standin) instead of
+    the prompt's queries, so that filling the cache skips the quadratic scoring pass."""
 
-    def __init__(self, w: synth.Workload, device, gen_device=None, hidden_seqs=None, prompt_layers=None):
+    def __init__(self, w: synth.Workload, device, gen_device=None, hidden_seqs=None, prompt_layers=None,
+                 standin_scores=False):
         self.w = w
         gen_device = gen_device or device
         self.hidden_seqs = w.batch if hidden_seqs is None else int(hidden_seqs)
@@ -41,7 +44,8 @@ class ResidentInputs:
             raise ValueError("hidden_seqs must divide the batch")
         self.hidden_repeat = w.batch // self.hidden_seqs
         n_pl = w.n_layer if prompt_layers is None else max(1, min(int(prompt_layers), w.n_layer))
-        need_q = w.policy == synth.H2O
+        need_q = w.policy == synth.H2O and not standin_scores
+        self.acc = None
 
         def place(t):
             out = _empty(t.shape, t.dtype, device)
@@ -57,6 +61,8 @@ class ResidentInputs:
             q, k, v = synth.prompt_qkv(w, l, gen_device, need_q=need_q)
             self._prompt.append((None if q is None else place(q), place(k), place(v)))
             del q, k, v
+        if w.policy == synth.H2O and standin_scores:
+            self.acc = [place(synth.prompt_scores_standin(w, l, gen_device)) for l in range(n_pl)]
         L, Bt, d = w.n_layer, w.batch, w.head_dim
         self.q = _empty((w.steps, L, Bt, w.n_q_head, d), w.dtype, device)
         self.k_new = _empty((w.steps, L, Bt, w.n_kv_head, d), w.dtype, device)
@@ -68,6 +74,9 @@ class ResidentInputs:
 
     def prompt(self, layer):
         return self._prompt[layer % len(self._prompt)]
+
+    def scores(self, layer):
+        return None if self.acc is None else self.acc[layer % len(self.acc)]
 
     def bytes_per_pass(self):
         """Bytes a pass fed from here moves: every distinct tensor once (a layer's hidden chunk is
@@ -104,7 +113,7 @@ class Job:
         ctx.allocate_budgets(w.b_init, w.p)
         for l in range(w.n_layer):
             q, k, v = inp.prompt(l)
-            ctx.prefill_compress(l, k, v, q)
+            ctx.prefill_compress(l, k, v, q, inp.scores(l))
 
     def decode(self, inp: ResidentInputs, steps=None):
         w, ctx = self.w, self.ctx
@@ -142,7 +151,8 @@ class Job:
         w = self.w
         per_layer = self.per_layer_decode if per_layer_decode is None else per_layer_decode
         h2o = w.policy == synth.H2O
-        per_layer_prefill = (2 + 1 + 1 + 1) if h2o else 1   # scores x2, select, gather, first victim
+        # H2O: two scoring sweeps (unless stand-in scores are given), selection, gather, first victim
+        per_layer_prefill = ((0 if inp.acc is not None else 2) + 1 + 1 + 1) if h2o else 1
         groups = w.n_layer if per_layer else 1
         per_step = groups * (2 if h2o else 1)
         return w.n_layer * inp.hidden_repeat + 1 + w.n_layer * per_layer_prefill + w.steps * per_step
@@ -153,6 +163,8 @@ class Job:
         a side stream overlapped with the kernels) and every step's output is copied back into
         out_host[t % len(out_host)]."""
         w, ctx, dev = self.w, self.ctx, self.device
+        if host.acc is not None:
+            raise ValueError("run_from_host computes the prompt scores from the prompt's queries")
         if not hasattr(self, "_stage"):
             a, b = host.hidden[0]
             q, k, v = host.prompt(0)

@@ -86,8 +86,13 @@ def falcon_7b(batch=32, prompt=2048, budget_pct=20.0, policy=SLIDING_WINDOW) -> 
                     heavy_mode="zipf" if policy == H2O else "none")
 
 
+def falcon_7b_max(policy=SLIDING_WINDOW) -> Workload:
+    """The largest cell of the Falcon-shaped sweep: batch 224, prompt 16384, budget 50 %."""
+    return falcon_7b(224, 16384, 50.0, policy)
+
+
 WORKLOADS = {"tiny": tiny, "llama2_7b": llama2_7b, "mistral_7b": mistral_7b,
-             "llama2_70b": llama2_70b, "falcon_7b": falcon_7b}
+             "llama2_70b": llama2_70b, "falcon_7b": falcon_7b, "falcon_7b_max": falcon_7b_max}
 
 
 def _gen(w: Workload, family: int, a: int = 0, b: int = 0, device="cpu") -> torch.Generator:
@@ -194,6 +199,18 @@ def prompt_qkv(w: Workload, layer: int, device="cpu", need_q=True):
     g = _gen(w, 3, layer, device=device)
     v = torch.randn(B, w.n_kv_head, P, d, generator=g, device=device, dtype=torch.float32).to(w.dtype)
     return q, k, v
+
+
+def prompt_scores_standin(w: Workload, layer: int, device="cpu"):
+    """Stand-in for a layer's accumulated prompt attention, fp32 [B, H_kv, P], for runs that fill
+    a cache without paying for the quadratic scoring pass: uniform draws scaled to the number of
+    query heads, with the heavy-hitter positions lifted well above the rest."""
+    g = _gen(w, 7, layer, device=device)
+    acc = torch.rand(w.batch, w.n_kv_head, w.prompt, generator=g, device=device, dtype=torch.float32) * w.group
+    for h, pos in enumerate(heavy_positions(w, layer)):
+        if pos.numel():
+            acc[:, h, pos.to(device)] += 50.0 * w.group
+    return acc
 
 
 def decode_qkv(w: Workload, step: int, device="cpu"):
