@@ -114,6 +114,19 @@ int sq_begin_sequence_batch(sq_ctx* ctx, int32_t batch, int32_t prompt_len, void
 int sq_layer_importance(sq_ctx* ctx, int32_t layer, const void* hidden_in, const void* hidden_out,
                         int64_t n_tok_total, void* stream);
 
+/* The same statistic taken where the hidden state after self-attention is made (Section 4.1:
+ * the similarities are collected "whenever the self-attention is conducted"; Table 4 prices the
+ * separate pass at +6.3 % of prefill).  resid: the residual stream entering the layer's
+ * attention block = the hidden state before self-attention; attn_out: the attention block's
+ * output; both [n_tok_total, hidden].  Writes hidden_out = resid + attn_out (one fp32 addition
+ * per element, rounded to the context's dtype) and adds the cosine between resid and that stored
+ * sum, token by token, to the layer's statistic: per token it reads 2 rows and writes 1, where a
+ * producer's own addition followed by sq_layer_importance reads 4 and writes 1.  hidden_out may
+ * be resid or attn_out itself (every element is read before it is written).  Chunking, call order
+ * and errors as for sq_layer_importance; the two calls may be mixed between layers. */
+int sq_layer_importance_fused(sq_ctx* ctx, int32_t layer, const void* resid, const void* attn_out, void* hidden_out,
+                              int64_t n_tok_total, void* stream);
+
 /* Algorithm 1, steps 5-12, and Appendix A.2.  Averages each layer's statistic, clusters the
  * n_layer averages (exact one-dimensional k-means with n_cluster groups; the group with the
  * largest average is the least important, G3), sets G3's budget to max(1, floor(b_init * p))

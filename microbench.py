@@ -1,6 +1,6 @@
 """Decode-step micro-benchmark: times sq_decode_step alone on any workload shape.
 
-    python -m paper_2404_04793_b200.microbench --workload falcon_7b --batch 32 --prompt 8192 \
+    python microbench.py --workload falcon_7b --batch 32 --prompt 8192 \
         --budget-pct 30 --policy sliding_window --steps 12 [--per-layer]
 
 The cache is filled through the regular calls (importance on a 256-token slice per layer,
@@ -15,7 +15,12 @@ import json
 
 import torch
 
-from . import engine, synth
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2404_04793_b200 import engine, synth  # noqa: E402
 
 POLICIES = {"sliding_window": synth.SLIDING_WINDOW, "streaming_llm": synth.STREAMING_LLM, "h2o": synth.H2O}
 

@@ -24,7 +24,7 @@ _ERR_NAMES = {1: "SQ_ERR_INVALID_ARG", 2: "SQ_ERR_STATE", 3: "SQ_ERR_CAPACITY", 
 
 # every symbol include/sq.h declares
 EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequence_batch",
-           "sq_layer_importance", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
+           "sq_layer_importance", "sq_layer_importance_fused", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
            "sq_decode_step", "sq_evict", "sq_get_cos_sim", "sq_get_budgets", "sq_get_kept", "sq_get_kv",
            "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static"]
 
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
     L.sq_ctx_destroy.argtypes = [P]
     L.sq_begin_sequence_batch.argtypes = [P, c_int32, c_int32, P]
     L.sq_layer_importance.argtypes = [P, c_int32, P, P, c_int64, P]
+    L.sq_layer_importance_fused.argtypes = [P, c_int32, P, P, P, c_int64, P]
     L.sq_allocate_budgets.argtypes = [P, c_int64, c_double, P]
     L.sq_set_budgets.argtypes = [P, POINTER(c_int32), P]
     L.sq_prefill_compress.argtypes = [P, c_int32, P, P, P, P, P]
@@ -155,6 +156,11 @@ class Context:
     def layer_importance(self, layer, hidden_in, hidden_out):
         n_tok = hidden_in.numel() // self.cfg.hidden
         self._ck(lib().sq_layer_importance(self._h, layer, _dptr(hidden_in), _dptr(hidden_out), n_tok, _stream()))
+
+    def layer_importance_fused(self, layer, resid, attn_out, hidden_out):
+        n_tok = resid.numel() // self.cfg.hidden
+        self._ck(lib().sq_layer_importance_fused(self._h, layer, _dptr(resid), _dptr(attn_out), _dptr(hidden_out), n_tok,
+                                                 _stream()))
 
     def allocate_budgets(self, b_init, p):
         self._ck(lib().sq_allocate_budgets(self._h, int(b_init), float(p), _stream()))

@@ -455,36 +455,15 @@ static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
   }
 }
 
-// Which attention kernel serves a shape: grouped bf16 heads go to the tensor-core kernel,
-// everything else (fp32, one query head per KV head, shapes it does not cover) to the fp32-pipe
-// kernel.  SQ_DECODE_PATH=alu|mma overrides the choice (mma also keeps wide groups off the tcgen05 kernel) (for A/B measurements).
-int decode_path_override() {
-  static int mode = -1;
-  if (mode < 0) {
-    const char* e = getenv("SQ_DECODE_PATH");
-    mode = !e ? 0 : (!strcmp(e, "alu") ? 1 : (!strcmp(e, "mma") ? 2 : 0));
-  }
-  return mode;
-}
-
-// SQ_H2O_UPDATE=cta keeps the H2O score update of unsplit launches on the CTA-per-unit kernel
-// (for A/B measurements).
-static bool h2o_update_override() {
-  static int mode = -1;
-  if (mode < 0) {
-    const char* e = getenv("SQ_H2O_UPDATE");
-    mode = (e && !strcmp(e, "cta")) ? 1 : 0;
-  }
-  return mode == 1;
-}
-
+// Which attention kernel serves a shape: wide bf16 groups at head_dim 64 go to the tcgen05
+// kernel, other grouped bf16 heads to the mma.sync kernel, everything else (fp32, one query head
+// per KV head, shapes those do not cover) to the fp32-pipe kernel.
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
-                          size_t q_rows, cudaStream_t s) {
+                          size_t q_rows, const int* desc_tiles, cudaStream_t s) {
   if (n_items <= 0) return cudaSuccess;
-  const int ovr = decode_path_override();
   bool done = false;
-  if (dtype == SQ_BF16 && ovr == 0 && a.group > 32) {
-    cudaError_t e = launch_decode_attn_tc(a, n_items, pool_bytes, q_rows, s);
+  if (dtype == SQ_BF16 && a.group > 32) {
+    cudaError_t e = launch_decode_attn_tc(a, desc_tiles, pool_bytes, q_rows, s);
     if (e == cudaSuccess) {
       // H2O: the attention kernel left the row log-sum-exps; the scores and the next victim come
       // from a second pass over K instead of logits carried through memory
@@ -497,7 +476,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   // every other kernel needs the per-slot logits for H2O: a context sized for the tcgen05 pair
   // does not hold them, and nothing may fall back silently
   if (!done && a.policy == SQ_POLICY_H2O && !a.has_logits) return cudaErrorNotSupported;
-  if (!done && dtype == SQ_BF16 && ovr != 1 && (a.group > 1 || ovr == 2)) {
+  if (!done && dtype == SQ_BF16 && a.group > 1) {
     cudaError_t e = launch_decode_attn_mma(a, n_items, s);
     if (e == cudaSuccess) done = true;
     else if (e != cudaErrorNotSupported) return e;
@@ -516,7 +495,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   // More units than the CTA-per-unit kernel holds in one wave (5 CTAs per SM), and nothing to
   // merge: only the scores and the next victim remain, one warp per unit.  Smaller launches
   // (one layer of a small batch) finish sooner with a CTA per unit.
-  if (a.policy == SQ_POLICY_H2O && a.uniform && a.group <= 32 && n_cta > 148 * 5 && !h2o_update_override()) {
+  if (a.policy == SQ_POLICY_H2O && a.uniform && a.group <= 32 && n_cta > 148 * 5) {
     h2o_update_warp_kernel<<<(n_cta + kWarpUpdWarps - 1) / kWarpUpdWarps, 32 * kWarpUpdWarps, 0, s>>>(a);
     return cudaGetLastError();
   }

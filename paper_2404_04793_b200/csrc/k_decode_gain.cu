@@ -9,7 +9,7 @@
 // accumulator in tensor memory, so that a thread owns one token: its probabilities
 // p = exp2(s*scale - lse_h) are summed over the heads in registers (no shuffles, no atomics,
 // head order fixed: deterministic), and the score read-modify-write is one coalesced access.
-//   warp 0      TMA: Q once, K tiles into a ring of stages (128-byte swizzle, no multicast)
+//   warp 0      TMA: Q once, K tiles into a ring of stages (128-byte swizzle, every CTA its own tiles)
 //   warp 1      MMA issue into a ring of accumulator buffers (three when the head columns fit
 //               three times into 256 tensor-memory columns, else two)
 //   warps 2..9  thread = one token (TMEM lane); warps 2..5 take the even tiles, warps 6..9 the

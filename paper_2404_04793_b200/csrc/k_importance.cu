@@ -9,7 +9,10 @@ namespace sq {
 // (A.B, A.A, B.B) in fp32 registers, and adds the token's cosine to the warp's running sum.
 // CTA sums go to cta_partial; the CTA that finishes last adds them up in index order (fp64),
 // so the result does not depend on scheduling.
-template <typename T>
+// FUSED: the rows are the residual stream (a) and the attention block's output (b); the kernel
+// writes their sum, rounded to T, to sum_out and takes the cosine between a and that sum, i.e.
+// between the hidden state before and after self-attention, in the pass that produces the latter.
+template <typename T, bool FUSED>
 __global__ void __launch_bounds__(256) cos_sim_reduce_kernel(ImportanceArgs a) {
   constexpr int EPV = Elem<T>::kPerVec;
   const int nvec = a.hidden / EPV;
@@ -19,6 +22,7 @@ __global__ void __launch_bounds__(256) cos_sim_reduce_kernel(ImportanceArgs a) {
   for (long long row = (long long)blockIdx.x * 8 + warp; row < a.n_tok; row += n_warp) {
     const uint4* pa = reinterpret_cast<const uint4*>(a.a) + row * nvec;
     const uint4* pb = reinterpret_cast<const uint4*>(a.b) + row * nvec;
+    uint4* po = FUSED ? reinterpret_cast<uint4*>(a.sum_out) + row * nvec : nullptr;
     float dot = 0.f, na = 0.f, nb = 0.f;
     for (int v0 = lane; v0 < nvec; v0 += 128) {
       uint4 va[4], vb[4];
@@ -38,6 +42,16 @@ __global__ void __launch_bounds__(256) cos_sim_reduce_kernel(ImportanceArgs a) {
         float fa[EPV], fb[EPV];
         widen<T>(va[u], fa);
         widen<T>(vb[u], fb);
+        if (FUSED) {
+          // the sum as it is stored: one fp32 addition, rounded to T
+          T r[EPV];
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) {
+            r[e] = narrow<T>(fa[e] + fb[e]);
+            fb[e] = to_float<T>(r[e]);
+          }
+          if (v0 + 32 * u < nvec) po[v0 + 32 * u] = *reinterpret_cast<const uint4*>(r);
+        }
 #pragma unroll
         for (int e = 0; e < EPV; ++e) {
           dot = fmaf(fa[e], fb[e], dot);
@@ -79,10 +93,13 @@ __global__ void __launch_bounds__(256) cos_sim_reduce_kernel(ImportanceArgs a) {
 }
 
 cudaError_t launch_importance(const ImportanceArgs& a, int dtype, int n_cta, cudaStream_t s) {
-  if (dtype == SQ_F32)
-    cos_sim_reduce_kernel<float><<<n_cta, 256, 0, s>>>(a);
-  else
-    cos_sim_reduce_kernel<__nv_bfloat16><<<n_cta, 256, 0, s>>>(a);
+  if (a.sum_out) {
+    if (dtype == SQ_F32) cos_sim_reduce_kernel<float, true><<<n_cta, 256, 0, s>>>(a);
+    else cos_sim_reduce_kernel<__nv_bfloat16, true><<<n_cta, 256, 0, s>>>(a);
+  } else {
+    if (dtype == SQ_F32) cos_sim_reduce_kernel<float, false><<<n_cta, 256, 0, s>>>(a);
+    else cos_sim_reduce_kernel<__nv_bfloat16, false><<<n_cta, 256, 0, s>>>(a);
+  }
   return cudaGetLastError();
 }
 

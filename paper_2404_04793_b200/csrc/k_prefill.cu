@@ -168,14 +168,9 @@ cudaError_t launch_prefill_scores_alu(const ScoreArgs& a, int dtype, cudaStream_
 }
 
 // bf16 prompts go to the tcgen05 kernels; fp32 (and anything those cannot serve) stays on the
-// fp32 pipes.  SQ_PREFILL_PATH=alu forces the latter (for A/B measurements).
+// fp32 pipes.
 cudaError_t launch_prefill_scores(const ScoreArgs& a, int dtype, int* status, cudaStream_t s) {
-  static int force_alu = -1;
-  if (force_alu < 0) {
-    const char* e = getenv("SQ_PREFILL_PATH");
-    force_alu = (e && !strcmp(e, "alu")) ? 1 : 0;
-  }
-  if (dtype == SQ_BF16 && !force_alu) {
+  if (dtype == SQ_BF16) {
     cudaError_t e = launch_prefill_scores_tc(a, status, s);
     if (e != cudaErrorNotSupported) return e;
   }

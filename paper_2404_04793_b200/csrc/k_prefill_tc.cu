@@ -11,7 +11,7 @@
 //     query tiles from the diagonal down and all heads of the group; thread t owns one key and
 //     adds exp2(s*scale - lse[row]) over the tile's columns -> the key's column sum, with no
 //     cross-thread reduction and no atomics (deterministic).
-// Roles per CTA (6 warps): warp 0 issues TMA tile loads (128-byte swizzle, no multicast) into
+// Roles per CTA (6 warps): warp 0 issues TMA tile loads (128-byte swizzle, every CTA its own tiles) into
 // a ring of shared-memory stages; warp 1 allocates tensor memory and issues the MMAs, signalling
 // completion through tcgen05.commit -> mbarrier; warps 2-5 drain the accumulators with
 // tcgen05.ld.  Two accumulator buffers let the next tile's MMA run under this tile's exponentials.

@@ -103,11 +103,10 @@ int check_config(const sq_config* c, std::string* why) {
 }
 
 // H2O decode of 33..128 bf16 query heads per KV head at head_dim 64 runs on the tcgen05 attention
-// + score-pass pair, which keeps no per-slot logits (SQ_DECODE_PATH forces the other kernels).
+// + score-pass pair, which keeps no per-slot logits.
 bool wide_h2o_pair(const sq_config& c) {
   const int G = c.n_q_head / c.n_kv_head;
-  return c.policy == SQ_POLICY_H2O && c.dtype == SQ_BF16 && c.head_dim == 64 && G > 32 && G <= kMaxGroup &&
-         decode_path_override() == 0;
+  return c.policy == SQ_POLICY_H2O && c.dtype == SQ_BF16 && c.head_dim == 64 && G > 32 && G <= kMaxGroup;
 }
 
 size_t pool_bytes_for(const sq_config& c, int64_t b_init) {
@@ -352,12 +351,13 @@ int sq_begin_sequence_batch(sq_ctx* c, int32_t batch, int32_t prompt_len, void* 
   return SQ_OK;
 }
 
-int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const void* hidden_out, int64_t n_tok_total,
-                        void* stream) {
+// Shared body of sq_layer_importance (sum_out null) and sq_layer_importance_fused.
+static int importance_rows(sq_ctx* c, int32_t layer, const void* row_a, const void* row_b, void* sum_out, int64_t n_tok_total,
+                           void* stream) {
   if (!c) return SQ_ERR_INVALID_ARG;
   if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
   if (layer < 0 || layer >= c->cfg.n_layer) return fail(c, SQ_ERR_INVALID_ARG, "layer out of range");
-  if (!hidden_in || !hidden_out || !aligned16(hidden_in) || !aligned16(hidden_out))
+  if (!row_a || !row_b || !aligned16(row_a) || !aligned16(row_b) || !aligned16(sum_out))
     return fail(c, SQ_ERR_INVALID_ARG, "hidden state pointers must be non-NULL and 16-byte aligned");
   if (n_tok_total < 0) return fail(c, SQ_ERR_INVALID_ARG, "n_tok_total is negative");
   if (n_tok_total == 0) return SQ_OK;
@@ -377,8 +377,9 @@ int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const v
     }
     const int d = layer * c->n_grp + grp;
     ImportanceArgs a;
-    a.a = static_cast<const char*>(hidden_in) + (size_t)done * row;
-    a.b = static_cast<const char*>(hidden_out) + (size_t)done * row;
+    a.a = static_cast<const char*>(row_a) + (size_t)done * row;
+    a.b = static_cast<const char*>(row_b) + (size_t)done * row;
+    a.sum_out = sum_out ? static_cast<char*>(sum_out) + (size_t)done * row : nullptr;
     a.n_tok = n;
     a.hidden = c->cfg.hidden;
     a.cta_partial = ws_ptr<float>(c, c->wl.cta_partial);
@@ -393,6 +394,17 @@ int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const v
   c->imp_tokens[layer] += n_tok_total;
   c->importance_seen[layer] = true;
   return SQ_OK;
+}
+
+int sq_layer_importance(sq_ctx* c, int32_t layer, const void* hidden_in, const void* hidden_out, int64_t n_tok_total,
+                        void* stream) {
+  return importance_rows(c, layer, hidden_in, hidden_out, nullptr, n_tok_total, stream);
+}
+
+int sq_layer_importance_fused(sq_ctx* c, int32_t layer, const void* resid, const void* attn_out, void* hidden_out,
+                              int64_t n_tok_total, void* stream) {
+  if (c && !hidden_out) return fail(c, SQ_ERR_INVALID_ARG, "hidden_out is NULL");
+  return importance_rows(c, layer, resid, attn_out, hidden_out, n_tok_total, stream);
 }
 
 int sq_allocate_budgets(sq_ctx* c, int64_t b_init, double p, void* stream) {
@@ -560,10 +572,6 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     int split = 0;
     double best_cost = 0.0;
     int prev = -1;
-    static const int forced = [] {  // SQ_SPLIT_PIECES=n forces n pieces per longest unit (for measurements)
-      const char* ev = getenv("SQ_SPLIT_PIECES");
-      return ev ? atoi(ev) : 0;
-    }();
     for (int pieces = 1; pieces <= (d1 - d0 > kMaxLayers ? 1 : 64); ++pieces) {
       int cand = ((max_len + pieces - 1) / pieces + tile - 1) / tile * tile;
       if (pieces > 1 && cand < 2 * tile) break;  // a piece is never shorter than two tiles
@@ -583,7 +591,7 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
       const double t_max = setup + (double)std::min(cand, max_len) / tile;
       const double spread = (double)work / (double)slots + 0.5 * t_max;
       const double cost = items <= slots ? t_max : std::max(t_max, std::min(spread, (double)waves * t_max));
-      if (forced > 0 ? (pieces <= forced) : (split == 0 || cost < best_cost * 0.90)) {  // more pieces only for a clear gain
+      if (split == 0 || cost < best_cost * 0.90) {  // more pieces only for a clear gain
         best_cost = cost;
         split = cand;
       }
@@ -632,8 +640,13 @@ int sq_decode_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const void
     a.policy = cfg.policy;
     a.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg.head_dim));
     const bool combine = cfg.policy == SQ_POLICY_H2O;  // other policies merge split-K pieces in the last piece
+    // 128-token tiles per unit of every descriptor, in launch order (the wide-group kernel deals
+    // the launch's tiles out evenly over the SMs)
+    std::vector<int> desc_tiles(d1 - d0);
+    for (int k = 0; k < d1 - d0; ++k)
+      desc_tiles[k] = (std::min(n_tok + 1, c->hs.layers[order_host[k]].b) + 127) / 128;
     SQ_CUDA(c, launch_decode(a, cfg.dtype, (int)n_items, combine, c->pool_bytes,
-                             (size_t)(e - s) * c->batch * cfg.n_q_head, st));
+                             (size_t)(e - s) * c->batch * cfg.n_q_head, desc_tiles.data(), st));
     for (int l = s; l < e; ++l) c->n_tok[l] += 1;
     s = e;
   }

@@ -34,6 +34,7 @@ __host__ __device__ inline int ring_slot(int x, int b, int base, int origin) {
 struct ImportanceArgs {
   const void* a;
   const void* b;
+  void* sum_out;         // fused form: receives a + b (rounded to the dtype), which then plays the part of b; else null
   long long n_tok;
   int hidden;
   float* cta_partial;    // [n_cta]
@@ -125,12 +126,12 @@ cudaError_t launch_select_prompt(const float* acc_prompt, int n_unit, int prompt
                                  int units_per_desc, char* pool, cudaStream_t s);
 cudaError_t launch_pick_victim(char* pool, const LayerDesc* descs, int units_per_desc, int n_unit, int prompt,
                                int next_pos, cudaStream_t s);
+// desc_tiles: per descriptor of the launch (launch order) the 128-token tiles of one unit
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
-                          size_t q_rows, cudaStream_t s);
-cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
+                          size_t q_rows, const int* desc_tiles, cudaStream_t s);
+cudaError_t launch_decode_attn_tc(const DecodeArgs& a, const int* desc_tiles, size_t pool_bytes, size_t q_rows, cudaStream_t s);
 cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
 cudaError_t launch_decode_attn_mma(const DecodeArgs& a, int n_items, cudaStream_t s);
 cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s);
-int decode_path_override();  // SQ_DECODE_PATH: 0 none, 1 alu, 2 mma
 
 }  // namespace sq

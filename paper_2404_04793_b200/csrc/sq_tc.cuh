@@ -1,5 +1,5 @@
 // PTX wrappers for the Blackwell tensor-core path: mbarriers with bounded waits, TMA tile loads
-// (no multicast), tcgen05 MMA / commit / tensor-memory loads and stores, shared-memory matrix
+// (every CTA loads its own tiles), tcgen05 MMA / commit / tensor-memory loads and stores, shared-memory matrix
 // descriptors for 128-byte-swizzled operand tiles.
 #pragma once
 #include <cuda.h>

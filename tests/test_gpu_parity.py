@@ -35,6 +35,50 @@ def test_layer_importance_matches_oracle(dtype, hidden, batch, prompt, chunks):
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("hidden,batch,prompt,chunks,in_place", [(128, 1, 256, 1, False), (4096, 2, 301, 3, False),
+                                                                 (4544, 3, 67, 2, True)])
+def test_fused_importance_matches_oracle_and_the_two_call_form(dtype, hidden, batch, prompt, chunks, in_place):
+    """The statistic taken in the pass that forms the hidden state after self-attention: the
+    stored sum is the dtype-rounded residual + attention output, the cosines are those of the
+    oracle on (residual, stored sum), and the budgets are bit for bit those of the separate call."""
+    w = small("impf", 12, hidden=hidden, batch=batch, prompt=prompt, dtype=dtype, n_layer=4)
+    fused, plain = H.make_ctx(w), H.make_ctx(w)
+    fused.begin_sequence_batch(w.batch, w.prompt)
+    plain.begin_sequence_batch(w.batch, w.prompt)
+    want = []
+    for l in range(w.n_layer):
+        resid, after = synth.hidden_pair(w, l, DEV)
+        resid, after = resid.reshape(-1, hidden), after.reshape(-1, hidden)
+        attn = (after.float() - resid.float()).to(dtype)                 # what the attention block adds
+        stored = (resid.float() + attn.float()).to(dtype)                # one fp32 addition, rounded
+        n = resid.shape[0]
+        edges = [round(i * n / chunks) for i in range(chunks + 1)]
+        out = torch.full_like(resid, float("nan"))
+        for i in range(chunks):
+            a, b = resid[edges[i]:edges[i + 1]].contiguous(), attn[edges[i]:edges[i + 1]].contiguous()
+            if in_place:
+                fused.layer_importance_fused(l, a, b, b)                 # the sum overwrites the attention output
+                out[edges[i]:edges[i + 1]] = b
+            else:
+                o = out[edges[i]:edges[i + 1]]
+                fused.layer_importance_fused(l, a, b, o)
+            assert torch.equal(a, resid[edges[i]:edges[i + 1]])          # inputs other than the target are untouched
+            plain.layer_importance(l, a, stored[edges[i]:edges[i + 1]].contiguous())   # same chunks: same summation order
+        torch.cuda.synchronize()
+        assert torch.equal(out, stored)
+        want.append(O.layer_importance(H.f64(resid), H.f64(stored)))
+    fused.allocate_budgets(w.b_init, w.p)
+    plain.allocate_budgets(w.b_init, w.p)
+    got = fused.get_cos_sim().numpy()
+    assert np.max(np.abs(got - np.array(want))) <= H.TOL_OUT[dtype]
+    assert np.array_equal(got, plain.get_cos_sim().numpy())
+    assert fused.get_budgets() == plain.get_budgets()
+    wb, wg = O.allocate_budgets(got, w.b_init, w.p)
+    assert fused.get_budgets() == (wb.tolist(), wg.tolist())
+    assert fused.status() == 0
+
+
 def test_layer_importance_special_vectors():
     w = small("imp2", 12, n_layer=4, hidden=64, batch=1, prompt=8)
     ctx = H.make_ctx(w)
