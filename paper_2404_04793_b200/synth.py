@@ -47,9 +47,12 @@ class Workload:
     heavy_num: int = 1
     heavy_den: int = 2
     heavy_mode: str = "none"  # "uniform4" | "zipf" | "none"
+    budget_tokens: int = 0    # > 0: the initial per-layer budget in absolute tokens (budget_pct is then unused)
 
     @property
     def b_init(self) -> int:
+        if self.budget_tokens > 0:
+            return int(self.budget_tokens)
         return int(math.floor(self.budget_pct * self.prompt / 100.0))
 
     @property
@@ -86,13 +89,23 @@ def falcon_7b(batch=32, prompt=2048, budget_pct=20.0, policy=SLIDING_WINDOW) -> 
                     heavy_mode="zipf" if policy == H2O else "none")
 
 
+def mistral_7b_long_generation(batch=32) -> Workload:
+    """Mistral-7B-shaped, the paper's throughput shape (prompt 512, 1024 generated tokens, Sliding
+    Window), with the budget given in absolute tokens, above the prompt length: 600 per layer.
+    The important layers' caches (about 1040 tokens) keep growing for some 530 steps before
+    their first eviction; the others (210 tokens) are compressed already at prefill."""
+    return Workload(f"mistral_7b_sw_p512_t1024_abs600_b{batch}", 6, 32, 32, 8, 128, 4096, batch, 512, 1024,
+                    torch.bfloat16, SLIDING_WINDOW, 0.0, 0.35, budget_tokens=600)
+
+
 def falcon_7b_max(policy=SLIDING_WINDOW) -> Workload:
     """The largest cell of the Falcon-shaped sweep: batch 224, prompt 16384, budget 50 %."""
     return falcon_7b(224, 16384, 50.0, policy)
 
 
 WORKLOADS = {"tiny": tiny, "llama2_7b": llama2_7b, "mistral_7b": mistral_7b,
-             "llama2_70b": llama2_70b, "falcon_7b": falcon_7b, "falcon_7b_max": falcon_7b_max}
+             "llama2_70b": llama2_70b, "falcon_7b": falcon_7b, "falcon_7b_max": falcon_7b_max,
+             "mistral_7b_long_generation": mistral_7b_long_generation}
 
 
 def _gen(w: Workload, family: int, a: int = 0, b: int = 0, device="cpu") -> torch.Generator:

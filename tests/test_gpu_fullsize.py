@@ -157,6 +157,15 @@ def test_falcon_7b_h2o_cell_lockstep_all_steps():
     _lockstep(synth.falcon_7b(32, 8192, 50.0, synth.H2O), n_units=16, steps=128, every_layer=False)
 
 
+def test_mistral_7b_absolute_budget_generation_longer_than_prompt():
+    """Budgets in absolute tokens above the prompt length (600 per layer for a 512-token prompt)
+    and 1024 generated tokens: the important layers' caches grow for hundreds of steps, reach
+    their budgets and evict from then on; the oracle follows every one of the 1024 steps."""
+    w = synth.mistral_7b_long_generation(batch=32)
+    assert w.b_init == 600 > w.prompt and w.steps == 1024
+    _follow(w, n_units=10, steps=w.steps, every_layer=False)
+
+
 def test_falcon_7b_mqa_cells():
     for policy, batch, prompt, pct in [(synth.SLIDING_WINDOW, 32, 2048, 20.0), (synth.STREAMING_LLM, 8, 8192, 10.0),
                                        (synth.H2O, 2, 2048, 30.0)]:
