@@ -47,7 +47,7 @@ DEFAULT_WORKLOAD = "falcon_7b_max"
 # DRAM bytes (read + write) per byte of K/V a decode launch has to read, from ncu captures of each
 # decode kernel on a small case (traffic grows in proportion to the units processed, each unit's
 # K/V being read once); None once a kernel has changed since its counters were taken.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"decode_attn_kernel": 1.008, "decode_attn_tc_kernel": None,
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"decode_attn_kernel": 1.008, "decode_attn_tc_kernel": 1.029,
                                     "decode_attn_mma_kernel": None}
 
 

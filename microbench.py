@@ -297,12 +297,12 @@ def main():
         compare_budgets()
         return
     if args.sweep_falcon:
-        for policy in ("sliding_window", "streaming_llm", "h2o"):
+        for policy in ([args.policy] if args.policy else ["sliding_window", "streaming_llm", "h2o"]):
             for batch in (1, 8, 32, 128, 224):
                 for prompt in (512, 2048, 8192, 16384):
                     for pct in (10.0, 20.0, 30.0, 50.0):
                         w = synth.falcon_7b(batch, prompt, pct, POLICIES[policy])
-                        r = decode_step_time(w, args.steps, args.warmup)
+                        r = decode_step_time(w, args.steps, args.warmup, args.per_layer)
                         r.update(policy=policy, batch=batch, prompt=prompt, budget_pct=pct)
                         print(json.dumps(r), flush=True)
                         torch.cuda.empty_cache()

@@ -33,6 +33,7 @@
 // tcgen05.ld/st, the tile redone): every weight stays finite and the result is that of the
 // exact softmax.  Every barrier wait is bounded.
 #include <algorithm>
+#include <type_traits>
 
 #include "sq_decode_common.cuh"
 #include "sq_internal.h"
@@ -381,9 +382,11 @@ __global__ void __launch_bounds__(192, kCtasPerSm)
     // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
     // (fp32 for the H2O normaliser, bf16-rounded for the output) to *sum / *sum_w; returns an
     // upper bound of the largest weight.
-    auto tile_weights = [&](int n_valid, float* sum, float* sum_w) {
+    // FULL (a compile-time tag): every token of the tile is valid, so no masking code is emitted
+    // (with a run-time flag the compare / select pair ran for every weight of every tile).
+    auto tile_weights = [&](auto full_tag, int n_valid, float* sum, float* sum_w) {
+      constexpr bool full = decltype(full_tag)::value;
       float acc = 0.f, acc_w = 0.f;
-      const bool full = (n_valid == kTM);
       auto chunk = [&](const uint32_t (&r)[32], int c) {
         uint32_t pk[16];
 #pragma unroll
@@ -447,7 +450,11 @@ __global__ void __launch_bounds__(192, kCtasPerSm)
         if (warp_live) {
           if (i == 0) m_ref = tile_max(n_valid);
           float sum, sum_w;
-          float pmax = tile_weights(n_valid, &sum, &sum_w);
+          auto weights = [&]() {
+            return (n_valid == kTM) ? tile_weights(std::true_type{}, n_valid, &sum, &sum_w)
+                                    : tile_weights(std::false_type{}, n_valid, &sum, &sum_w);
+          };
+          float pmax = weights();
           if (__any_sync(0xffffffffu, pmax > kMaxWeight)) {
             // rare: move the reference of the rows that need it; O and the sums (complete up to
             // the previous tile) shrink with it, then the tile is redone.  The whole warp takes
@@ -469,7 +476,7 @@ __global__ void __launch_bounds__(192, kCtasPerSm)
             l_true *= f;
             l_w *= f;
             if (need) m_ref = mx2;
-            pmax = tile_weights(n_valid, &sum, &sum_w);
+            pmax = weights();
           }
           l_true += sum;
           l_w += sum_w;
