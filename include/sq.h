@@ -22,7 +22,9 @@
  *     aligned, of the context's dtype unless stated.  "host" pointers are marked.
  *   - The library allocates no device memory.  The caller provides one cache pool and one
  *     workspace (sizes from sq_query_sizes); both must stay valid until sq_ctx_destroy and
- *     must not be touched by the caller in between.
+ *     must not be touched by the caller in between.  sq_ctx_create allocates one small block of
+ *     page-locked HOST memory (staging of the budget and layout tables, a few KB per layer) and
+ *     one CUDA event; sq_ctx_destroy frees them.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
  *     enqueued on it and calls return without waiting, except the sq_get_* calls and
  *     sq_status, which synchronise the device, and the first call after sq_allocate_budgets
@@ -188,6 +190,29 @@ int sq_get_len(sq_ctx* ctx, int32_t layer, int32_t* len);
 /* Device-side status word: 0 = clean; non-zero = a kernel detected an inconsistency. */
 int sq_status(sq_ctx* ctx, int32_t* device_status);
 const char* sq_last_error(sq_ctx* ctx);
+
+/* Checkpoint / resume.  The cache state of a batch is the caller's pool plus this table: one
+ * entry per layer (per (sequence, layer), sequence first, with per_sequence_budgets).  Offsets
+ * are bytes from the pool base; a unit's slots are rows [unit * cap, unit * cap + min(n_tok,
+ * budget)) of each region (K, V rows of head_dim elements; pos int32; acc fp32, H2O only; victim
+ * int32 per unit, H2O only).  To resume: copy the pool's bytes back (or keep the pool), create a
+ * context with the same config and b_init, sq_begin_sequence_batch with the same batch and
+ * prompt_len, then sq_ctx_import_layout with the exported table; decoding continues with the
+ * next token as if it had not stopped.  Export synchronises the device; import is host work plus
+ * small asynchronous copies on `stream` and one wait for them. */
+typedef struct sq_layer_layout {
+  int64_t k_off, v_off, pos_off, acc_off, victim_off;
+  int32_t budget;      /* tokens kept per unit                                              */
+  int32_t cap;         /* slots per unit (budget rounded up to page_tokens)                 */
+  int32_t b_heavy;     /* H2O: slots of the budget held for heavy hitters                   */
+  int32_t ring_base;   /* Sliding Window 0, StreamingLLM n_sink: slots below it never move  */
+  int32_t ring_origin; /* the position stored in slot ring_base                             */
+  int32_t n_tok;       /* tokens seen so far (prompt + generated); -1: layer not prefilled  */
+  int32_t n_unit;      /* units that share this entry                                       */
+  int32_t reserved;
+} sq_layer_layout;
+int sq_ctx_export_layout(sq_ctx* ctx, sq_layer_layout* layout_host /* [n_layer]; [batch][n_layer] with per_sequence_budgets */);
+int sq_ctx_import_layout(sq_ctx* ctx, const sq_layer_layout* layout_host, void* stream);
 
 /* Bytes of K+V the decode kernel reads per step for the given layer range at the current
  * fill level (for bandwidth accounting). */

@@ -245,6 +245,39 @@ def generation_throughput(w: synth.Workload, device="cuda:0"):
                 device_status=ctx.status())
 
 
+def importance_time(w: synth.Workload, reps=5, device="cuda:0", n_seq=4):
+    """Layer importance of one layer's hidden states (n_seq sequences of the workload's prompt
+    length): the separate pass over (hidden_in, hidden_out); the producer's own residual addition
+    (an elementwise kernel) followed by that pass; and the fused call that writes the sum and
+    takes the statistic in one pass."""
+    job = engine.Job(w.replace(steps=1, batch=n_seq), device)
+    ctx = job.ctx
+    ctx.begin_sequence_batch(n_seq, w.prompt)
+    a, b = synth.hidden_pair(w, 0, device, batch=n_seq)
+    attn = (b.float() - a.float()).to(w.dtype)
+    out = torch.empty_like(a)
+    nbytes = a.numel() * a.element_size()
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_sep = timed(lambda: ctx.layer_importance(0, a, b))
+    ms_two = timed(lambda: (torch.add(a, attn, out=out), ctx.layer_importance(0, a, out)))
+    ms_fused = timed(lambda: ctx.layer_importance_fused(0, a, attn, out))
+    return dict(workload=w.name, what="layer importance, one layer", tokens=n_seq * w.prompt, bytes_per_array=nbytes,
+                separate_pass_ms=round(ms_sep, 4), separate_pass_GBs=round(2 * nbytes / ms_sep / 1e6, 1),
+                add_then_pass_ms=round(ms_two, 4), add_then_pass_GBs=round(5 * nbytes / ms_two / 1e6, 1),
+                fused_ms=round(ms_fused, 4), fused_GBs=round(3 * nbytes / ms_fused / 1e6, 1), device_status=ctx.status())
+
+
 def compare_budgets():
     """Full cache vs a sequence-wise policy alone vs the layer-wise reallocation on the same
     kernels, on the shapes of the paper's throughput table (attention path only, no weights)."""
@@ -278,6 +311,7 @@ def main():
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--per-sequence", action="store_true", help="per-sequence budgets (a rotated budget vector per sequence)")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
+    ap.add_argument("--importance", action="store_true", help="time sq_layer_importance, separate and fused with the residual addition")
     ap.add_argument("--evict", action="store_true", help="time one explicit eviction of all layers to half the budgets")
     ap.add_argument("--all-kernels", action="store_true", help="launch every kernel of the library once or a few times")
     ap.add_argument("--layers", type=int, default=0, help="with --all-kernels: number of layers of the shape to keep")
@@ -306,6 +340,9 @@ def main():
                         r.update(policy=policy, batch=batch, prompt=prompt, budget_pct=pct)
                         print(json.dumps(r), flush=True)
                         torch.cuda.empty_cache()
+        return
+    if args.importance:
+        print(json.dumps(importance_time(build_workload(args), args.steps)), flush=True)
         return
     if args.prefill:
         print(json.dumps(prefill_compress_time(build_workload(args), args.steps)), flush=True)

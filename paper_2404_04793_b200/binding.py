@@ -26,7 +26,8 @@ _ERR_NAMES = {1: "SQ_ERR_INVALID_ARG", 2: "SQ_ERR_STATE", 3: "SQ_ERR_CAPACITY", 
 EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequence_batch",
            "sq_layer_importance", "sq_layer_importance_fused", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
            "sq_decode_step", "sq_evict", "sq_get_cos_sim", "sq_get_budgets", "sq_get_kept", "sq_get_kv",
-           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static"]
+           "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static",
+           "sq_ctx_export_layout", "sq_ctx_import_layout"]
 
 
 class sq_config(ctypes.Structure):
@@ -34,6 +35,11 @@ class sq_config(ctypes.Structure):
         "n_layer", "n_q_head", "n_kv_head", "head_dim", "hidden", "max_batch", "max_prompt",
         "max_new_tokens", "dtype", "policy", "n_sink", "heavy_num", "heavy_den", "n_cluster", "page_tokens",
         "per_sequence_budgets")]
+
+
+class sq_layer_layout(ctypes.Structure):
+    _fields_ = [(n, c_int64) for n in ("k_off", "v_off", "pos_off", "acc_off", "victim_off")] + \
+               [(n, c_int32) for n in ("budget", "cap", "b_heavy", "ring_base", "ring_origin", "n_tok", "n_unit", "reserved")]
 
 
 class SqError(RuntimeError):
@@ -75,6 +81,8 @@ def lib() -> ctypes.CDLL:
     L.sq_last_error.argtypes = [P]
     L.sq_last_error.restype = c_char_p
     L.sq_kv_bytes_per_step.argtypes = [P, c_int32, c_int32, POINTER(c_int64)]
+    L.sq_ctx_export_layout.argtypes = [P, POINTER(sq_layer_layout)]
+    L.sq_ctx_import_layout.argtypes = [P, POINTER(sq_layer_layout), P]
     L.sq_prompt_scores_static.argtypes = [P, P, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, P, P]
     for name in EXPORTS:
         if name != "sq_last_error":
@@ -133,6 +141,7 @@ class Context:
             raise SqError(rc, "sq_ctx_create")
         self._h = h
         self.pool_bytes, self.workspace_bytes = pool_bytes, ws_bytes
+        self.pool_view = self.pool[po:po + pool_bytes]     # the bytes the library was given
 
     def close(self):
         if getattr(self, "_h", None):
@@ -235,6 +244,16 @@ class Context:
         v = torch.empty(max(cap, 1), self.cfg.head_dim, dtype=dt)
         self._ck(lib().sq_get_kv(self._h, layer, seq, kv_head, c_void_p(k.data_ptr()), c_void_p(v.data_ptr())))
         return k[:n], v[:n]
+
+    def export_layout(self):
+        """The cache geometry and fill level per layer (ctypes array, C layout): with a copy of
+        `pool` it is the whole state of the batch."""
+        arr = (sq_layer_layout * (self.cfg.n_layer * self._rows()))()
+        self._ck(lib().sq_ctx_export_layout(self._h, arr))
+        return arr
+
+    def import_layout(self, layout):
+        self._ck(lib().sq_ctx_import_layout(self._h, layout, _stream()))
 
     def status(self):
         s = c_int32()

@@ -463,7 +463,9 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need
   if (n_items <= 0) return cudaSuccess;
   bool done = false;
   if (dtype == SQ_BF16 && a.group > 32) {
-    cudaError_t e = launch_decode_attn_tc(a, desc_tiles, pool_bytes, q_rows, s);
+    // long units that do not fill the CTA slots: the even deal; else one CTA per unit and piece
+    cudaError_t e = launch_decode_attn_tc_stream(a, desc_tiles, pool_bytes, q_rows, s);
+    if (e == cudaErrorNotSupported) e = launch_decode_attn_tc(a, n_items, pool_bytes, q_rows, s);
     if (e == cudaSuccess) {
       // H2O: the attention kernel left the row log-sum-exps; the scores and the next victim come
       // from a second pass over K instead of logits carried through memory

@@ -849,6 +849,71 @@ int sq_status(sq_ctx* c, int32_t* device_status) {
   return SQ_OK;
 }
 
+int sq_ctx_export_layout(sq_ctx* c, sq_layer_layout* out) {
+  if (!c || !out) return SQ_ERR_INVALID_ARG;
+  if (c->budget_state != 2) return fail(c, SQ_ERR_STATE, "budgets not laid out yet");
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    for (int g = 0; g < c->n_grp; ++g) {
+      const LayerDesc& ld = c->hs.layers[l * c->n_grp + g];
+      sq_layer_layout& o = out[user_index(c, l, g)];
+      o.k_off = ld.k_off;
+      o.v_off = ld.v_off;
+      o.pos_off = ld.pos_off;
+      o.acc_off = ld.acc_off;
+      o.victim_off = ld.victim_off;
+      o.budget = ld.b;
+      o.cap = ld.cap;
+      o.b_heavy = ld.b_heavy;
+      o.ring_base = ld.ring_base;
+      o.ring_origin = ld.ring_origin;
+      o.n_tok = c->prefilled[l] ? c->n_tok[l] : -1;
+      o.n_unit = c->desc_units;
+      o.reserved = 0;
+    }
+  return SQ_OK;
+}
+
+int sq_ctx_import_layout(sq_ctx* c, const sq_layer_layout* in, void* stream) {
+  if (!c || !in) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (c->budget_state == 1) SQ_CUDA(c, cudaEventSynchronize(c->ev));
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    for (int g = 0; g < c->n_grp; ++g) {
+      const sq_layer_layout& e = in[user_index(c, l, g)];
+      if (e.n_unit != c->desc_units) return fail(c, SQ_ERR_INVALID_ARG, "layout was exported for another batch shape");
+      if (e.n_tok != in[user_index(c, l, 0)].n_tok) return fail(c, SQ_ERR_INVALID_ARG, "sequences of a layer disagree on n_tok");
+      c->hs.budget[l * c->n_grp + g] = e.budget;
+      c->hs.is_g3[l * c->n_grp + g] = 0;
+    }
+  c->budget_state = 0;
+  int rc = build_layout(c, st);  // the geometry these budgets give in this context's pool
+  if (rc != SQ_OK) return rc;
+  for (int l = 0; l < c->cfg.n_layer; ++l) {
+    for (int g = 0; g < c->n_grp; ++g) {
+      const sq_layer_layout& e = in[user_index(c, l, g)];
+      LayerDesc& ld = c->hs.layers[l * c->n_grp + g];
+      if (e.k_off != ld.k_off || e.v_off != ld.v_off || e.pos_off != ld.pos_off || e.acc_off != ld.acc_off ||
+          e.victim_off != ld.victim_off || e.cap != ld.cap || e.b_heavy != ld.b_heavy || e.ring_base != ld.ring_base) {
+        c->budget_state = 0;
+        return fail(c, SQ_ERR_INVALID_ARG, "layout does not match this context's config, b_init or pool");
+      }
+      ld.ring_origin = e.ring_origin;  // moves with explicit evictions
+    }
+    const int n_tok = in[user_index(c, l, 0)].n_tok;
+    c->prefilled[l] = n_tok >= 0;
+    c->n_tok[l] = n_tok >= 0 ? n_tok : 0;
+    if (n_tok > c->cfg.max_prompt + c->cfg.max_new_tokens) return fail(c, SQ_ERR_INVALID_ARG, "n_tok beyond the context's limits");
+  }
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers), c->hs.layers, sizeof(LayerDesc) * c->n_desc,
+                             cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs.budget, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemsetAsync(ws_ptr<unsigned char>(c, c->wl.is_g3), 0, c->n_desc, st));
+  SQ_CUDA(c, cudaStreamSynchronize(st));
+  return SQ_OK;
+}
+
 int sq_kv_bytes_per_step(sq_ctx* c, int32_t layer_begin, int32_t layer_end, int64_t* bytes) {
   if (!c || !bytes) return SQ_ERR_INVALID_ARG;
   if (layer_begin < 0 || layer_end > c->cfg.n_layer || layer_begin >= layer_end)

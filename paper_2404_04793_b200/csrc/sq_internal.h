@@ -129,7 +129,9 @@ cudaError_t launch_pick_victim(char* pool, const LayerDesc* descs, int units_per
 // desc_tiles: per descriptor of the launch (launch order) the 128-token tiles of one unit
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int n_items, bool need_combine, size_t pool_bytes,
                           size_t q_rows, const int* desc_tiles, cudaStream_t s);
-cudaError_t launch_decode_attn_tc(const DecodeArgs& a, const int* desc_tiles, size_t pool_bytes, size_t q_rows, cudaStream_t s);
+cudaError_t launch_decode_attn_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
+cudaError_t launch_decode_attn_tc_stream(const DecodeArgs& a, const int* desc_tiles, size_t pool_bytes, size_t q_rows,
+                                         cudaStream_t s);
 cudaError_t launch_h2o_gain_tc(const DecodeArgs& a, int n_items, size_t pool_bytes, size_t q_rows, cudaStream_t s);
 cudaError_t launch_decode_attn_mma(const DecodeArgs& a, int n_items, cudaStream_t s);
 cudaError_t launch_evict(const EvictArgs& a, cudaStream_t s);

@@ -42,6 +42,19 @@ def test_config_struct_matches_the_header():
     assert ctypes.sizeof(B.sq_config) == 4 * len(fields)
 
 
+def test_layout_struct_matches_the_header():
+    """The ctypes mirror of sq_layer_layout lists the header's fields in the header's order and width."""
+    text = open(os.path.join(ROOT, "include", "sq.h")).read()
+    body = text[text.index("typedef struct sq_layer_layout {"):text.index("} sq_layer_layout;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = []
+    for ctype, names in re.findall(r"(int64_t|int32_t)\s+([a-z_, ]+);", body):
+        fields += [(n.strip(), ctype) for n in names.split(",")]
+    mirror = [(n, "int64_t" if t is ctypes.c_int64 else "int32_t") for n, t in B.sq_layer_layout._fields_]
+    assert fields == mirror
+    assert ctypes.sizeof(B.sq_layer_layout) == 5 * 8 + 8 * 4
+
+
 def test_per_sequence_budgets_size_the_tables(lib):
     """One descriptor per (layer, sequence): the workspace grows with the batch, the K/V part of the pool does not."""
     p0, w0 = B.sq_query_sizes(_cfg(max_batch=8), 100)

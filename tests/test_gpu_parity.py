@@ -446,6 +446,55 @@ def test_evict_of_a_growing_h2o_cache_to_exactly_its_length(dtype, head_dim, hq,
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("policy,dtype,head_dim,hq,hkv", [
+    (synth.SLIDING_WINDOW, torch.bfloat16, 128, 4, 4), (synth.STREAMING_LLM, torch.bfloat16, 128, 8, 2),
+    (synth.H2O, torch.float32, 64, 4, 2), (synth.H2O, torch.bfloat16, 64, 71, 1)])
+def test_checkpoint_and_resume_through_the_exported_layout(policy, dtype, head_dim, hq, hkv):
+    """A batch stopped after some steps (one explicit eviction among them) and resumed in a fresh
+    context from the exported layout table and a copy of the pool's bytes continues bit for bit
+    like the batch that was never stopped."""
+    w = small("ckpt", 28, policy=policy, dtype=dtype, head_dim=head_dim, n_q_head=hq, n_kv_head=hkv,
+              heavy_mode="uniform4", steps=10)
+    budgets = [40, 30, 120]
+
+    def fresh():
+        ctx = H.make_ctx(w, b_init=max(budgets))
+        ctx.begin_sequence_batch(w.batch, w.prompt)
+        return ctx
+
+    def step(ctx, t):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, w.n_layer, q, kn, vn, out)
+        return out
+
+    a = fresh()
+    a.set_budgets(budgets)
+    H.prefill_all(a, w, DEV, keep_inputs=False)
+    for t in range(3):
+        step(a, t)
+    a.evict(0, w.n_layer, [25, 30, 64])
+    step(a, 3)
+    layout = a.export_layout()
+    assert [e.budget for e in layout] == [25, 30, 64] and all(e.n_tok == w.prompt + 4 for e in layout)
+    saved = a.pool_view.clone()
+    b = fresh()
+    b.import_layout(layout)
+    b.pool_view.copy_(saved)
+    assert b.get_budgets()[0] == [25, 30, 64]
+    for t in range(4, w.steps):
+        oa, ob = step(a, t), step(b, t)
+        assert torch.equal(oa, ob), t
+    for key in H.all_units(w):
+        assert a.get_kept(*key) == b.get_kept(*key)
+    assert a.status() == 0 and b.status() == 0
+    # a table from another shape is refused
+    other = H.make_ctx(w.replace(batch=w.batch + 1), b_init=max(budgets))
+    other.begin_sequence_batch(w.batch + 1, w.prompt)
+    with pytest.raises(B.SqError):
+        other.import_layout(layout)
+
+
 # ----------------------------------------------------------------- error paths
 def test_call_order_and_argument_errors():
     w = small("err", 26)
