@@ -199,11 +199,14 @@ const char* sq_last_error(sq_ctx* ctx);
  * context with the same config and b_init, sq_begin_sequence_batch with the same batch and
  * prompt_len, then sq_ctx_import_layout with the exported table; decoding continues with the
  * next token as if it had not stopped.  Export synchronises the device; import is host work plus
- * small asynchronous copies on `stream` and one wait for them. */
+ * small asynchronous copies on `stream` and one wait for them.  Import lays the pool out by the
+ * table's capacities and returns SQ_ERR_INVALID_ARG, changing nothing the caller can decode
+ * from, when the table's offsets are not the ones this context gives those capacities. */
 typedef struct sq_layer_layout {
   int64_t k_off, v_off, pos_off, acc_off, victim_off;
   int32_t budget;      /* tokens kept per unit                                              */
-  int32_t cap;         /* slots per unit (budget rounded up to page_tokens)                 */
+  int32_t cap;         /* slots per unit: the budget the layer was laid out with, rounded
+                          up to page_tokens (an explicit eviction lowers budget, not cap)   */
   int32_t b_heavy;     /* H2O: slots of the budget held for heavy hitters                   */
   int32_t ring_base;   /* Sliding Window 0, StreamingLLM n_sink: slots below it never move  */
   int32_t ring_origin; /* the position stored in slot ring_base                             */

@@ -6,17 +6,28 @@
 //   O[head rows x 64]        += P V_tile         (P bf16 in TENSOR memory, V tile MN-major)
 // One CTA per (layer, unit, split), two CTAs per SM; per 128-token tile the roles are
 //   warp 0      TMA: K and V tiles into a ring of stages (128-byte swizzle, every CTA its own tiles)
-//   warp 1      MMA issue
+//   warp 1      MMA issue (one thread)
 //   warps 2..5  thread = one head row (TMEM lane): p = exp2(s*scale - m_ref) straight from the
 //               accumulator row, no shuffles; P is packed to bf16 and stored back to tensor
 //               memory as the A operand of the second MMA
 // Measured on B200: one M=128, K=16 MMA costs 45-48 cycles for N <= 64 and 64 cycles for N = 128,
 // and operands read from shared memory compete with the TMA writes for its 128 B/clk; keeping P
-// in tensor memory (64 columns) removes 56 KB of shared-memory traffic per tile.
+// in tensor memory (64 columns) removes 56 KB of shared-memory traffic per tile.  Inside the
+// kernel, two CTAs sharing the pipe, an MMA holds the issuing thread for about 80 cycles and a
+// tcgen05.commit for about 180.
 // A row's reference m_ref is its maximum over the first tile; later tiles reuse it and only
 // when a weight would exceed 2^16 is the reference moved (O and the sums rescaled through
 // tcgen05.ld/st, the tile redone): every weight stays finite and the result is that of the
 // exact softmax.  Every barrier wait is bounded.
+// What bounds the kernel (measured on B200 with per-tile clock stamps and with copies that leave
+// work out): a softmax warp needs 1250 cycles per tile alone on its scheduler and 2150-2250 when
+// it shares it with the other CTA's (the special-function unit: 128 exp2 per row and tile at one
+// warp instruction per 8 cycles), against 2780 cycles of HBM time per pair of tiles at 1.9 GHz;
+// a polynomial exp2 on the FMA pipe for a part of the weights was slower at every share tried.
+// Streaming K and V alone (no products, no softmax) reaches 7.3 TB/s and draws 970 W of the
+// board's 1000 W; with the products 6.4 TB/s, with the softmax as well 4.6-4.7 TB/s, both at the
+// power limit with the SM clock near 1.5-1.6 GHz: run for longer than a few milliseconds the
+// kernel is bound by power, and what helps is fewer instructions per weight.
 #include <type_traits>
 
 #include "sq_decode_common.cuh"
@@ -159,34 +170,31 @@ __global__ void __launch_bounds__(192, 2)
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    const uint32_t q_addr = s_u32(q_s);
-    auto issue_s = [&](int i) -> bool {
-      const int st = i % STAGES;
-      if (!mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag)) return false;
-      if (i >= 1 && !mbar_wait(bar_sfree, (i - 1) & 1, abort_flag)) return false;
-      tc_fence_after();
-      if (lane == 0) {
+    // ---------------- MMA issuer: one thread ----------------
+    if (lane == 0) {
+      const uint32_t q_addr = s_u32(q_s);
+      auto issue_s = [&](int i) -> bool {
+        const int st = i % STAGES;
+        if (!mbar_wait(bar_full(st), (i / STAGES) & 1, abort_flag)) return false;
+        if (i >= 1 && !mbar_wait(bar_sfree, (i - 1) & 1, abort_flag)) return false;
+        tc_fence_after();
         const uint32_t k_addr = s_u32(k_s + st * kTileBytes);
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k)
           umma_bf16(tmem_base + kColS, umma_desc(q_addr + k * 32), umma_desc(k_addr + k * 32), idesc(128, false),
                     k > 0 ? 1u : 0u);
         umma_commit(bar_sfull);
-      }
-      __syncwarp();
-      return true;
-    };
-    bool ok = mbar_wait(bar_q, 0, abort_flag);
-    if (ok) ok = issue_s(0);
-    for (int i = 0; ok && i < n_tiles; ++i) {
-      if (i + 1 < n_tiles) ok = issue_s(i + 1);
-      if (!ok) break;
-      const int st = i % STAGES;
-      ok = mbar_wait(bar_pready, i & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      if (lane == 0) {
+        return true;
+      };
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      if (ok) ok = issue_s(0);
+      for (int i = 0; ok && i < n_tiles; ++i) {
+        if (i + 1 < n_tiles) ok = issue_s(i + 1);
+        if (!ok) break;
+        const int st = i % STAGES;
+        ok = mbar_wait(bar_pready, i & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
         const uint32_t v_addr = s_u32(v_s + st * kTileBytes);
 #pragma unroll
         for (int k = 0; k < kTM / 16; ++k)
@@ -197,8 +205,8 @@ __global__ void __launch_bounds__(192, 2)
         umma_commit(bar_pfree);
         umma_commit(bar_odone);
       }
-      __syncwarp();
     }
+    __syncwarp();
   } else {
     // ---------------- softmax: thread = one head row ----------------
     const int quarter = warp & 3;
@@ -208,7 +216,7 @@ __global__ void __launch_bounds__(192, 2)
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
     const uint32_t s_addr = tmem_base + lane_sel + kColS, p_addr = tmem_base + lane_sel + kColP,
                    o_addr = tmem_base + lane_sel + kColO;
-    float m_ref = -INFINITY, l_true = 0.f, l_w = 0.f;
+    float m_ref = -INFINITY, l = 0.f, l_w = 0.f;  // the row's reference; sums of its weights, exact and as rounded to bf16
     bool ok = true;
 
     // Row maximum of the tile's valid tokens, in the log2 domain.
@@ -225,29 +233,41 @@ __global__ void __launch_bounds__(192, 2)
       return mx * a.scale_log2;
     };
     // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
-    // (fp32 for the H2O normaliser, bf16-rounded for the output) to *sum / *sum_w; returns an
-    // upper bound of the largest weight.
+    // (exact fp32 for the H2O normaliser, of the bf16-rounded weights for the output) to *sum /
+    // *sum_w; returns an upper bound of the largest weight.  The role is bound by the
+    // special-function unit (one exp2 per 8 cycles per warp) and by the issue slots of one or two
+    // softmax warps per scheduler, so the scaling runs as packed fp32x2 instructions and the
+    // rounded weights are summed by mixed-precision adds: six instructions per two weights.
     // FULL (a compile-time tag): every token of the tile is valid, so no masking code is emitted
     // (with a run-time flag the compare / select pair ran for every weight of every tile).
-    auto tile_weights = [&](auto full_tag, int n_valid, float* sum, float* sum_w) {
+    auto tile_weights = [&](auto full_tag, int n_valid, float* sum, float* sum_w, bool* s_released) {
       constexpr bool full = decltype(full_tag)::value;
-      float acc = 0.f, acc_w = 0.f;
+      const unsigned long long scale2 = f32x2(a.scale_log2, a.scale_log2), neg_m2 = f32x2(-m_ref, -m_ref);
+      unsigned long long acc2 = f32x2(0.f, 0.f);  // exact sums (H2O), even and odd tokens
+      float w_a = 0.f, w_b = 0.f;                 // sums of the rounded weights
       auto chunk = [&](const uint32_t (&r)[32], int c) {
-        uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_ref));
-          if (!full) {
-            if (c * 32 + j >= n_valid) p0 = 0.f;
-            if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+        for (int hc = 0; hc < 2; ++hc) {  // P goes back sixteen tokens (eight columns) at a time
+          uint32_t pk[8];
+#pragma unroll
+          for (int jj = 0; jj < 16; jj += 2) {
+            const int j = hc * 16 + jj;
+            float p0, p1;
+            f32x2_split(fma_f32x2(f32x2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), scale2, neg_m2), p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
+            if (!full) {
+              if (c * 32 + j >= n_valid) p0 = 0.f;
+              if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+            }
+            if (H2O) acc2 = add_f32x2(acc2, f32x2(p0, p1));
+            const uint32_t u = pack2(p0, p1);  // round to nearest bf16, p0 in the low half
+            w_a = add_bf16_lo(w_a, u);
+            w_b = add_bf16_hi(w_b, u);
+            pk[jj / 2] = u;
           }
-          if (H2O) acc += p0 + p1;
-          const uint32_t u = pack2(p0, p1);  // round to nearest bf16, p0 in the low half
-          acc_w += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
-          pk[j / 2] = u;
+          tmem_st8_u32(p_addr + c * 16 + hc * 8, pk);  // tokens c*32 + hc*16 .. +15 of this row
         }
-        tmem_st16_u32(p_addr + c * 16, pk);  // tokens c*32 .. c*32+31 of this row
       };
       // the next chunk's tensor-memory load is in flight while this one is processed
       uint32_t ra[32], rb[32];
@@ -262,11 +282,30 @@ __global__ void __launch_bounds__(192, 2)
       tmem_ld32_nowait(s_addr + 96, rb);
       chunk(ra, 2);
       tmem_wait_ld(rb);
+      {
+        // The last quarter of S is in registers.  Unless the tile may have to be redone (the
+        // weights so far, or a logit of this quarter, too large), S is handed back now, so the
+        // tensor core computes the next tile's S while these 32 weights are worked out.
+        float mx = __uint_as_float(rb[0]);
+#pragma unroll
+        for (int j = 1; j + 1 < 32; j += 2) mx = max3(mx, __uint_as_float(rb[j]), __uint_as_float(rb[j + 1]));
+        mx = fmaxf(mx, __uint_as_float(rb[31]));
+        const float so_far = w_a + w_b;
+        // 32 weights of at most 2^10 and 2^15 before them stay below kMaxWeight
+        const bool safe = so_far <= 32768.f && fmaf(mx, a.scale_log2, -m_ref) <= 10.f;
+        *s_released = __all_sync(0xffffffffu, safe);
+        if (*s_released) {
+          tc_fence_before();
+          if (lane == 0) mbar_arrive(bar_sfree);
+        }
+      }
       chunk(rb, 3);
       tmem_wait_st();
-      *sum = acc;
-      *sum_w = acc_w;
-      return acc_w;  // the tile's weight sum bounds its largest weight
+      float s0, s1;
+      f32x2_split(acc2, s0, s1);
+      *sum = s0 + s1;
+      *sum_w = w_a + w_b;
+      return w_a + w_b;  // the tile's weight sum bounds its largest weight
     };
 
     for (int i = 0; ok && i < n_tiles; ++i) {
@@ -287,12 +326,13 @@ __global__ void __launch_bounds__(192, 2)
       }
       if (!ok) break;
       tc_fence_after();
+      bool s_released = false;
       if (warp_live) {
         if (i == 0) m_ref = tile_max(n_valid);
         float sum, sum_w;
         auto weights = [&]() {
-          return (n_valid == kTM) ? tile_weights(std::true_type{}, n_valid, &sum, &sum_w)
-                                  : tile_weights(std::false_type{}, n_valid, &sum, &sum_w);
+          return (n_valid == kTM) ? tile_weights(std::true_type{}, n_valid, &sum, &sum_w, &s_released)
+                                  : tile_weights(std::false_type{}, n_valid, &sum, &sum_w, &s_released);
         };
         float pmax = weights();
         if (__any_sync(0xffffffffu, pmax > kMaxWeight)) {
@@ -313,19 +353,19 @@ __global__ void __launch_bounds__(192, 2)
             for (int j = 0; j < 32; ++j) o[j] *= f;
             tmem_st32(o_addr + c * 32, o);
           }
-          l_true *= f;
+          l *= f;
           l_w *= f;
           if (need) m_ref = mx2;
           pmax = weights();
         }
-        l_true += sum;
+        l += sum;
         l_w += sum_w;
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(bar_pready);
-        mbar_arrive(bar_sfree);
+        if (!s_released) mbar_arrive(bar_sfree);
       }
     }
     // ---------------- epilogue: O / l -> out (or the split-K partial) ----------------
@@ -356,10 +396,10 @@ __global__ void __launch_bounds__(192, 2)
       }
       if (live) {
         stat[row * kStatStride] = m_ref;
-        stat[row * kStatStride + 1] = H2O ? l_true : l_w;
+        stat[row * kStatStride + 1] = H2O ? l : l_w;
         stat[row * kStatStride + 2] = l_w;
         // H2O: the unit's row log-sum-exps (log2 domain), read by the score-update pass that follows
-        if (H2O && it.n_split == 1) (a.logits + ldp->lse_off + (size_t)unit * G)[row] = m_ref + log2f(l_true);
+        if (H2O && it.n_split == 1) (a.logits + ldp->lse_off + (size_t)unit * G)[row] = m_ref + log2f(l);
       }
     }
   }

@@ -349,29 +349,41 @@ __global__ void __launch_bounds__(192, kCtasPerSm)
       return mx * a.scale_log2;
     };
     // p = exp2(s*scale - m_ref) for the whole tile: P (bf16) to tensor memory; sums of the weights
-    // (fp32 for the H2O normaliser, bf16-rounded for the output) to *sum / *sum_w; returns an
-    // upper bound of the largest weight.
+    // (exact fp32 for the H2O normaliser, of the bf16-rounded weights for the output) to *sum /
+    // *sum_w; returns an upper bound of the largest weight.  The role is bound by the
+    // special-function unit (one exp2 per 8 cycles per warp) and by the issue slots of one or two
+    // softmax warps per scheduler, so the scaling runs as packed fp32x2 instructions and the
+    // rounded weights are summed by mixed-precision adds: six instructions per two weights.
     // FULL (a compile-time tag): every token of the tile is valid, so no masking code is emitted
     // (with a run-time flag the compare / select pair ran for every weight of every tile).
     auto tile_weights = [&](auto full_tag, int n_valid, float* sum, float* sum_w) {
       constexpr bool full = decltype(full_tag)::value;
-      float acc = 0.f, acc_w = 0.f;
+      const unsigned long long scale2 = f32x2(a.scale_log2, a.scale_log2), neg_m2 = f32x2(-m_ref, -m_ref);
+      unsigned long long acc2 = f32x2(0.f, 0.f);
+      float w_a = 0.f, w_b = 0.f;
       auto chunk = [&](const uint32_t (&r)[32], int c) {
-        uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_ref));
-          if (!full) {
-            if (c * 32 + j >= n_valid) p0 = 0.f;
-            if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+        for (int hc = 0; hc < 2; ++hc) {  // P goes back sixteen tokens (eight columns) at a time
+          uint32_t pk[8];
+#pragma unroll
+          for (int jj = 0; jj < 16; jj += 2) {
+            const int j = hc * 16 + jj;
+            float p0, p1;
+            f32x2_split(fma_f32x2(f32x2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), scale2, neg_m2), p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
+            if (!full) {
+              if (c * 32 + j >= n_valid) p0 = 0.f;
+              if (c * 32 + j + 1 >= n_valid) p1 = 0.f;
+            }
+            if (H2O) acc2 = add_f32x2(acc2, f32x2(p0, p1));
+            const uint32_t u = pack2(p0, p1);  // round to nearest bf16, p0 in the low half
+            w_a = add_bf16_lo(w_a, u);
+            w_b = add_bf16_hi(w_b, u);
+            pk[jj / 2] = u;
           }
-          if (H2O) acc += p0 + p1;
-          const uint32_t u = pack2(p0, p1);  // round to nearest bf16, p0 in the low half
-          acc_w += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
-          pk[j / 2] = u;
+          tmem_st8_u32(p_addr + c * 16 + hc * 8, pk);  // tokens c*32 + hc*16 .. +15 of this row
         }
-        tmem_st16_u32(p_addr + c * 16, pk);  // tokens c*32 .. c*32+31 of this row
       };
       // the next chunk's tensor-memory load is in flight while this one is processed
       uint32_t ra[32], rb[32];
@@ -388,9 +400,11 @@ __global__ void __launch_bounds__(192, kCtasPerSm)
       tmem_wait_ld(rb);
       chunk(rb, 3);
       tmem_wait_st();
-      *sum = acc;
-      *sum_w = acc_w;
-      return acc_w;  // the tile's weight sum bounds its largest weight
+      float s0, s1;
+      f32x2_split(acc2, s0, s1);
+      *sum = s0 + s1;
+      *sum_w = w_a + w_b;
+      return w_a + w_b;  // the tile's weight sum bounds its largest weight
     };
 
     while (ok && it.next(a)) {

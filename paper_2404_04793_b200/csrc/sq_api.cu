@@ -877,40 +877,59 @@ int sq_ctx_export_layout(sq_ctx* c, sq_layer_layout* out) {
 int sq_ctx_import_layout(sq_ctx* c, const sq_layer_layout* in, void* stream) {
   if (!c || !in) return SQ_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const sq_config& cfg = c->cfg;
   if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
   if (c->budget_state == 1) SQ_CUDA(c, cudaEventSynchronize(c->ev));
-  for (int l = 0; l < c->cfg.n_layer; ++l)
+  // The geometry follows the slots a layer was laid out with, not its present budget (an explicit
+  // eviction lowers the budget and leaves the slots where they are): lay the pool out by the
+  // exported capacities, then put the budgets back.
+  for (int l = 0; l < cfg.n_layer; ++l)
     for (int g = 0; g < c->n_grp; ++g) {
       const sq_layer_layout& e = in[user_index(c, l, g)];
       if (e.n_unit != c->desc_units) return fail(c, SQ_ERR_INVALID_ARG, "layout was exported for another batch shape");
       if (e.n_tok != in[user_index(c, l, 0)].n_tok) return fail(c, SQ_ERR_INVALID_ARG, "sequences of a layer disagree on n_tok");
-      c->hs.budget[l * c->n_grp + g] = e.budget;
+      if (e.n_tok > cfg.max_prompt + cfg.max_new_tokens) return fail(c, SQ_ERR_INVALID_ARG, "n_tok beyond the context's limits");
+      if (e.cap < 1 || e.cap % cfg.page_tokens != 0 || e.budget < 1 || e.budget > e.cap)
+        return fail(c, SQ_ERR_INVALID_ARG, "layout: budget / cap");
+      if (cfg.policy == SQ_POLICY_STREAMING_LLM && e.budget <= cfg.n_sink)
+        return fail(c, SQ_ERR_INVALID_ARG, "StreamingLLM needs every layer budget above n_sink");
+      c->hs.budget[l * c->n_grp + g] = e.cap;
       c->hs.is_g3[l * c->n_grp + g] = 0;
     }
   c->budget_state = 0;
-  int rc = build_layout(c, st);  // the geometry these budgets give in this context's pool
+  int rc = build_layout(c, st);
   if (rc != SQ_OK) return rc;
-  for (int l = 0; l < c->cfg.n_layer; ++l) {
+  c->budget_state = 0;  // until the descriptors below are in place
+  for (int l = 0; l < cfg.n_layer; ++l) {
     for (int g = 0; g < c->n_grp; ++g) {
       const sq_layer_layout& e = in[user_index(c, l, g)];
-      LayerDesc& ld = c->hs.layers[l * c->n_grp + g];
+      const int d = l * c->n_grp + g;
+      LayerDesc& ld = c->hs.layers[d];
+      const int b_heavy = cfg.policy == SQ_POLICY_H2O ? (int)(((long long)e.budget * cfg.heavy_num) / cfg.heavy_den) : 0;
       if (e.k_off != ld.k_off || e.v_off != ld.v_off || e.pos_off != ld.pos_off || e.acc_off != ld.acc_off ||
-          e.victim_off != ld.victim_off || e.cap != ld.cap || e.b_heavy != ld.b_heavy || e.ring_base != ld.ring_base) {
-        c->budget_state = 0;
-        return fail(c, SQ_ERR_INVALID_ARG, "layout does not match this context's config, b_init or pool");
-      }
-      ld.ring_origin = e.ring_origin;  // moves with explicit evictions
+          e.victim_off != ld.victim_off || e.cap != ld.cap || e.b_heavy != b_heavy || e.ring_base != ld.ring_base)
+        return fail(c, SQ_ERR_INVALID_ARG, "layout does not match this context's config or pool");
+      if (e.ring_origin < ld.ring_base) return fail(c, SQ_ERR_INVALID_ARG, "layout: ring_origin");
+      ld.b = e.budget;
+      ld.b_heavy = b_heavy;
+      ld.b_recent = e.budget - b_heavy;
+      ld.ring_origin = e.ring_origin;  // moved by explicit evictions
+      c->hs.budget[d] = e.budget;
     }
     const int n_tok = in[user_index(c, l, 0)].n_tok;
     c->prefilled[l] = n_tok >= 0;
     c->n_tok[l] = n_tok >= 0 ? n_tok : 0;
-    if (n_tok > c->cfg.max_prompt + c->cfg.max_new_tokens) return fail(c, SQ_ERR_INVALID_ARG, "n_tok beyond the context's limits");
   }
+  sort_orders(c);
   SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<LayerDesc>(c, c->wl.layers), c->hs.layers, sizeof(LayerDesc) * c->n_desc,
+                             cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order), c->hs.order, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.order_by_layer), c->hs.order_by_layer, 4 * c->n_desc,
                              cudaMemcpyHostToDevice, st));
   SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<int>(c, c->wl.budget), c->hs.budget, 4 * c->n_desc, cudaMemcpyHostToDevice, st));
   SQ_CUDA(c, cudaMemsetAsync(ws_ptr<unsigned char>(c, c->wl.is_g3), 0, c->n_desc, st));
   SQ_CUDA(c, cudaStreamSynchronize(st));
+  c->budget_state = 2;
   return SQ_OK;
 }
 
