@@ -48,7 +48,7 @@ DEFAULT_WORKLOAD = "falcon_7b_max"
 # decode kernel on a small case (traffic grows in proportion to the units processed, each unit's
 # K/V being read once); None once a kernel has changed since its counters were taken.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = {"decode_attn_kernel": 1.008, "decode_attn_tc_kernel": 1.018,
-                                    "decode_attn_tc_stream_kernel": 1.036, "decode_attn_mma_kernel": None}
+                                    "decode_attn_tc_stream_kernel": 1.033, "decode_attn_mma_kernel": None}
 
 
 def workload_by_name(name):
