@@ -330,6 +330,47 @@ def test_decode_wide_mqa_growing_logits():
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("policy", [synth.SLIDING_WINDOW, synth.H2O])
+def test_decode_wide_mqa_even_deal_launch(policy):
+    """One layer of a batch whose units are long but fewer than the CTA slots goes to the kernel
+    that deals the launch's tiles out evenly: segments end inside units, so pieces are merged by
+    the last to arrive; a ragged last tile; and, for some sequences, keys that grow along the
+    cache, so that the softmax reference has to move inside a segment."""
+    w = small("mqa_deal", 31, policy=policy, dtype=torch.bfloat16, head_dim=64, n_q_head=71, n_kv_head=1,
+              batch=160, n_layer=1, prompt=2100, steps=2, hidden=64, heavy_mode="none")
+    b = 2200  # 18 tiles per unit, 160 units for 296 CTA slots; the cache is still growing
+    ctx = H.make_ctx(w, b_init=b)
+    ctx.begin_sequence_batch(w.batch, w.prompt)
+    ctx.set_budgets([b])
+    q_p, k, v = synth.prompt_qkv(w, 0, DEV, need_q=(policy == synth.H2O))
+    k = k.clone()
+    grow = [0, 7, 159]
+    for s_ in grow:
+        k[s_, :, 700:1400] *= 10.0
+        k[s_, :, 1400:] *= 25.0
+    ctx.prefill_compress(0, k, v, q_p)
+    seqs = [0, 1, 7, 80, 158, 159]
+    units = {}
+    for s_ in seqs:
+        u = O.UnitCache(policy, b, w.n_sink, w.heavy_num, w.heavy_den)
+        u.prefill(H.f64(k[s_, 0]), H.f64(v[s_, 0]), H.f64(q_p[s_]) if policy == synth.H2O else None)
+        units[s_] = u
+    for t in range(w.steps):
+        q, kn, vn = synth.decode_qkv(w, t, DEV)
+        out = torch.empty_like(q)
+        ctx.decode_step(0, 1, q[0], kn[0], vn[0], out[0])
+        for s_, u in units.items():
+            want = u.decode_step(H.f64(q[0, s_]), H.f64(kn[0, s_, 0]), H.f64(vn[0, s_, 0]))
+            got = H.f64(out[0, s_])
+            tol = np.maximum(H.TOL_OUT[w.dtype], 2.0 ** -7 * np.abs(want))
+            assert np.all(np.abs(got - want) <= tol), (t, s_, np.max(np.abs(got - want)))
+            if policy == synth.H2O:
+                pos, acc = ctx.get_kept(0, s_, 0)
+                assert pos == u.kept_positions()
+                assert np.allclose(acc, u.acc, rtol=H.RTOL_ACC[w.dtype], atol=1e-6), (t, s_)
+    assert ctx.status() == 0
+
+
 def test_decode_budget_one_and_sinks_only_edge():
     w = small("edge", 22, policy=synth.SLIDING_WINDOW, steps=3)
     _run_decode_and_compare(w, budgets=[1, 2, 3])
