@@ -114,7 +114,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.f.close()
-        sm, mx, reasons = [], [], set()
+        sm, mx, watts, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             p = [x.strip() for x in line.split(",")]
@@ -128,6 +128,10 @@ class ClockSampler:
                 sm.append(float(p[1])); mx.append(float(p[2]))
             except ValueError:
                 continue
+            try:
+                watts.append(float(p[3]))
+            except ValueError:
+                pass
             for n, v in zip(names, p[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
@@ -137,6 +141,8 @@ class ClockSampler:
             pass
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            if watts:
+                out["power_w"] = statistics.median(watts)
         return out
 
 

@@ -45,7 +45,8 @@ def build_workload(args) -> synth.Workload:
     return w
 
 
-def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, device="cuda:0", per_sequence=False):
+def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, device="cuda:0", per_sequence=False,
+                     sample_clocks=False):
     job = engine.Job(w.replace(steps=steps + warmup), device)
     ctx = job.ctx
     ctx.begin_sequence_batch(w.batch, w.prompt)
@@ -86,6 +87,16 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
         step()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = None
+    if sample_clocks:
+        # SM clock, power and throttle reasons while the timed steps run (a run of a second or
+        # more reaches the board's power limit; a few steps do not)
+        import time
+        from bench import ClockSampler
+        sampler = ClockSampler(torch.cuda.current_device())
+        sampler.start()
+        time.sleep(0.3)
+        t_begin = time.time()
     if per_layer:
         # one launch per layer is CPU-bound when issued from Python: time a CUDA-graph replay of
         # the same launches instead (kernel arguments frozen at capture; the caches are full, so
@@ -105,6 +116,7 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
             step()
         e1.record()
     torch.cuda.synchronize()
+    clocks = sampler.stop(t_begin, time.time()) if sampler else None
     ms = e0.elapsed_time(e1) / steps
     e = 2 if w.dtype == torch.bfloat16 else 4
     kv = int(w.batch * w.n_kv_head * sum(min(w.prompt + 1, b) for b in budgets) * 2 * w.head_dim * e)
@@ -113,7 +125,8 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
     gbs = (kv + io + extra) / ms / 1e6
     return dict(workload=w.name, per_layer=per_layer, per_sequence_budgets=per_sequence, ms_per_step=round(ms, 4), GBs=round(gbs, 1),
                 kv_GB=round(kv / 1e9, 3), algorithmic_bytes=kv + io + extra, tokens_per_s=round(w.batch / ms * 1e3),
-                flops=int(4 * w.n_q_head * w.head_dim * w.batch * sum(budgets)), device_status=ctx.status())
+                flops=int(4 * w.n_q_head * w.head_dim * w.batch * sum(budgets)), device_status=ctx.status(),
+                **({"clocks": clocks} if clocks else {}))
 
 
 def prefill_compress_time(w: synth.Workload, reps=3, device="cuda:0"):
@@ -309,6 +322,7 @@ def main():
     ap.add_argument("--steps", type=int, default=12)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--per-layer", action="store_true")
+    ap.add_argument("--sample-clocks", action="store_true", help="decode step: SM clock, power and throttle reasons during the timed steps")
     ap.add_argument("--per-sequence", action="store_true", help="per-sequence budgets (a rotated budget vector per sequence)")
     ap.add_argument("--prefill", action="store_true", help="time sq_prefill_compress of one layer instead")
     ap.add_argument("--importance", action="store_true", help="time sq_layer_importance, separate and fused with the residual addition")
@@ -351,7 +365,7 @@ def main():
         print(json.dumps(evict_time(build_workload(args), min(args.steps, 5))), flush=True)
         return
     print(json.dumps(decode_step_time(build_workload(args), args.steps, args.warmup, args.per_layer,
-                                      per_sequence=args.per_sequence)), flush=True)
+                                      per_sequence=args.per_sequence, sample_clocks=args.sample_clocks)), flush=True)
 
 
 if __name__ == "__main__":
