@@ -58,13 +58,15 @@ def workload_by_name(name):
     return synth.WORKLOADS[name]()
 
 
-def config_of(w, world):
+def config_of(w, world, shard_batch=False):
     """The workload as the JSON line names it (both arms print the same keys)."""
     from paper_2404_04793_b200 import synth
+    how = ("one batch sharded by sequence; one all-reduce of 2 x n_layer numbers per pass before the allocation"
+           if shard_batch else "independent batches")
     return {"workload": w.name, "n_layer": w.n_layer, "n_q_head": w.n_q_head, "n_kv_head": w.n_kv_head,
             "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch, "prompt": w.prompt,
             "decode_steps": w.steps, "policy": synth.POLICY_NAMES[w.policy], "b_init": w.b_init, "p": w.p,
-            "parallelism": f"dp{world} (independent batches)"}
+            "parallelism": f"dp{world} ({how})"}
 
 
 def maybe_spawn(argv, gpus):
@@ -495,11 +497,19 @@ def run_ours(args, w):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     peak, peak_kind = hbm_peak()
-    # every rank owns an independent batch: a different seed family per rank
+    # every rank owns an independent batch (a different seed family per rank); with --shard-batch
+    # the ranks hold the sequences of ONE batch, B / world each, and exchange the layer sums of the
+    # importance pass before the allocation, so that all of them get the batch's budgets
     wr = w.replace(wid=w.wid + 100 * rank) if world > 1 else w
+    exchange = None
+    if args.shard_batch:
+        if w.batch % world:
+            raise SystemExit("--shard-batch needs a batch divisible by the number of ranks")
+        wr = wr.replace(batch=w.batch // world)
+        exchange = lambda ctx: dist_util.exchange_importance(ctx, dev)
     hs = hidden_seqs_for(wr)
     inp = engine.ResidentInputs(wr, dev, hidden_seqs=hs)
-    job = engine.Job(wr, dev, per_layer_decode=True, keep_steps=min(wr.steps, 16))
+    job = engine.Job(wr, dev, per_layer_decode=True, keep_steps=min(wr.steps, 16), exchange=exchange)
     tokens = wr.batch * wr.steps
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -636,7 +646,7 @@ def run_ours(args, w):
         cpu = oracle_sample(wr, n_units=args.cpu_units, n_imp_tokens=16384, seed=7, device=dev,
                             pool_cores=cores if cores > 1 else 0)
 
-    cfg = config_of(wr, world)
+    cfg = config_of(wr, world, args.shard_batch)
     cfg.update({"budgets_min_max": [min(budgets), max(budgets)], "n_g3": int(sum(is_g3)),
                 "decode_launch": "per_layer (one launch per layer per step, CUDA-graph replay)",
                 "hidden_states": f"{hs} distinct sequences per layer, fed {hidden_repeat}x (every token's bytes are read)",
@@ -644,7 +654,7 @@ def run_ours(args, w):
                       % (kv_bytes / 1e9, kv_bytes / wr.n_layer / 1e6)})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "strong" if args.shard_batch else "weak", "vs_baseline": None,
         "dtype": "bf16" if wr.dtype == torch.bfloat16 else "f32", "data": "synthetic", "config": cfg,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
         "decode_only": {"tokens_per_s": tokens / (ms_decode * 1e-3), "ms_per_token_step": ms_decode / wr.steps,
@@ -667,6 +677,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps")
     ap.add_argument("--cpu-units", type=int, default=4, help="units the one-core oracle timing samples")
+    ap.add_argument("--shard-batch", action="store_true",
+                    help="--gpus N: one batch of the workload's size sharded over the ranks (strong scaling) instead of one batch per rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the fused-launch upper bound")
     ap.add_argument("--no-records", action="store_true", help="skip the decode-step records of the other configurations")

@@ -174,6 +174,17 @@ int sq_decode_step(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, const vo
 int sq_evict(sq_ctx* ctx, int32_t layer_begin, int32_t layer_end, const int32_t* new_budgets_host,
              void* stream);
 
+/* One batch sharded over several GPUs (each rank holds some of its sequences and their whole
+ * cache): with one budget vector for the batch, the layer averages of Section 3's cosine run over
+ * the tokens of all ranks, so the ranks exchange, once, after the last sq_layer_importance and
+ * before sq_allocate_budgets, the per-layer sums of cosines and token counts (2 * n_layer numbers;
+ * summed over the ranks by the caller, e.g. one all-reduce) and every rank then runs the same
+ * deterministic allocation.  sq_get_importance_state reads this context's sums (synchronises);
+ * sq_set_importance_state replaces them (host arrays [n_layer]; asynchronous on `stream`).  Not
+ * available with per_sequence_budgets (nothing to exchange there): SQ_ERR_UNSUPPORTED. */
+int sq_get_importance_state(sq_ctx* ctx, double* cos_sum_host /* [n_layer] */, int64_t* n_tok_host /* [n_layer] */);
+int sq_set_importance_state(sq_ctx* ctx, const double* cos_sum_host, const int64_t* n_tok_host, void* stream);
+
 /* Read-back (host outputs; these synchronise). */
 int sq_get_cos_sim(sq_ctx* ctx, float* cos_sim_host /* [n_layer]; [batch][n_layer] with per_sequence_budgets */);
 int sq_get_budgets(sq_ctx* ctx, int32_t* budgets_host /* same shape */, uint8_t* is_g3_host /* same shape, or NULL */);

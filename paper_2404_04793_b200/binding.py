@@ -27,7 +27,7 @@ EXPORTS = ["sq_query_sizes", "sq_ctx_create", "sq_ctx_destroy", "sq_begin_sequen
            "sq_layer_importance", "sq_layer_importance_fused", "sq_allocate_budgets", "sq_set_budgets", "sq_prefill_compress",
            "sq_decode_step", "sq_evict", "sq_get_cos_sim", "sq_get_budgets", "sq_get_kept", "sq_get_kv",
            "sq_get_len", "sq_status", "sq_last_error", "sq_kv_bytes_per_step", "sq_prompt_scores_static",
-           "sq_ctx_export_layout", "sq_ctx_import_layout"]
+           "sq_ctx_export_layout", "sq_ctx_import_layout", "sq_get_importance_state", "sq_set_importance_state"]
 
 
 class sq_config(ctypes.Structure):
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
     L.sq_decode_step.argtypes = [P, c_int32, c_int32, P, P, P, P, P]
     L.sq_evict.argtypes = [P, c_int32, c_int32, POINTER(c_int32), P]
     L.sq_get_cos_sim.argtypes = [P, POINTER(c_float)]
+    L.sq_get_importance_state.argtypes = [P, POINTER(c_double), POINTER(c_int64)]
+    L.sq_set_importance_state.argtypes = [P, POINTER(c_double), POINTER(c_int64), P]
     L.sq_get_budgets.argtypes = [P, POINTER(c_int32), POINTER(c_uint8)]
     L.sq_get_kept.argtypes = [P, c_int32, c_int32, c_int32, POINTER(c_int32), POINTER(c_float), POINTER(c_int32)]
     L.sq_get_kv.argtypes = [P, c_int32, c_int32, c_int32, P, P]
@@ -210,6 +212,19 @@ class Context:
         flat = self._flatten(new_budgets, layer_end - layer_begin)
         arr = (c_int32 * len(flat))(*flat)
         self._ck(lib().sq_evict(self._h, layer_begin, layer_end, arr, _stream()))
+
+    def get_importance_state(self):
+        """Per-layer sums of cosines and token counts accumulated so far (per-batch budgets)."""
+        n = self.cfg.n_layer
+        sums, counts = (c_double * n)(), (c_int64 * n)()
+        self._ck(lib().sq_get_importance_state(self._h, sums, counts))
+        return list(sums), list(counts)
+
+    def set_importance_state(self, sums, counts):
+        n = self.cfg.n_layer
+        a = (c_double * n)(*[float(x) for x in sums])
+        b = (c_int64 * n)(*[int(x) for x in counts])
+        self._ck(lib().sq_set_importance_state(self._h, a, b, _stream()))
 
     def get_cos_sim(self):
         arr = (c_float * (self.cfg.n_layer * self._rows()))()

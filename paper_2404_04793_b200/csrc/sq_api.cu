@@ -743,6 +743,32 @@ int sq_evict(sq_ctx* c, int32_t layer_begin, int32_t layer_end, const int32_t* n
   return SQ_OK;
 }
 
+int sq_get_importance_state(sq_ctx* c, double* cos_sum_host, int64_t* n_tok_host) {
+  if (!c || !cos_sum_host || !n_tok_host) return SQ_ERR_INVALID_ARG;
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (c->per_seq) return fail(c, SQ_ERR_UNSUPPORTED, "per-sequence budgets have no state to exchange");
+  SQ_CUDA(c, cudaDeviceSynchronize());
+  SQ_CUDA(c, cudaMemcpy(cos_sum_host, ws_ptr<double>(c, c->wl.cos_sum), 8 * c->cfg.n_layer, cudaMemcpyDeviceToHost));
+  for (int l = 0; l < c->cfg.n_layer; ++l) n_tok_host[l] = c->hs.tok_count[l];
+  return SQ_OK;
+}
+
+int sq_set_importance_state(sq_ctx* c, const double* cos_sum_host, const int64_t* n_tok_host, void* stream) {
+  if (!c || !cos_sum_host || !n_tok_host) return SQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->begun) return fail(c, SQ_ERR_STATE, "sq_begin_sequence_batch has not been called");
+  if (c->per_seq) return fail(c, SQ_ERR_UNSUPPORTED, "per-sequence budgets have no state to exchange");
+  for (int l = 0; l < c->cfg.n_layer; ++l)
+    if (n_tok_host[l] < 1) return fail(c, SQ_ERR_INVALID_ARG, "a layer's token count is below 1");
+  // pageable source: the copy has left the caller's array when the call returns
+  SQ_CUDA(c, cudaMemcpyAsync(ws_ptr<double>(c, c->wl.cos_sum), cos_sum_host, 8 * c->cfg.n_layer, cudaMemcpyHostToDevice, st));
+  for (int l = 0; l < c->cfg.n_layer; ++l) {
+    c->hs.tok_count[l] = n_tok_host[l];
+    c->importance_seen[l] = true;
+  }
+  return SQ_OK;
+}
+
 int sq_get_cos_sim(sq_ctx* c, float* cos_sim_host) {
   if (!c || !cos_sim_host) return SQ_ERR_INVALID_ARG;
   if (c->budget_state == 0) return fail(c, SQ_ERR_STATE, "sq_allocate_budgets has not been called");

@@ -43,6 +43,22 @@ def sum_over_ranks(value: float, device="cpu") -> float:
     return float(t.item())
 
 
+def exchange_importance(ctx, device="cpu"):
+    """One batch sharded over the ranks (each holds some of its sequences): sums the per-layer
+    cosine sums and token counts of Section 3's layer average over all ranks (one all-reduce of
+    2 * n_layer numbers) and puts the totals back into this rank's context, so that
+    allocate_budgets gives every rank the batch's budgets.  Call after the last layer_importance."""
+    sums, counts = ctx.get_importance_state()
+    if dist.is_initialized():
+        t = torch.tensor(list(sums) + [float(c) for c in counts], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        v = t.cpu().tolist()
+        n = len(sums)
+        sums, counts = v[:n], [int(round(x)) for x in v[n:]]
+    ctx.set_importance_state(sums, counts)
+    return sums, counts
+
+
 def aggregate_throughput(units_this_rank: float, ms_this_rank: float, device="cpu"):
     """Whole-job throughput: units processed by all ranks / the slowest rank's time.
     Returns (units_per_second, max_ms)."""

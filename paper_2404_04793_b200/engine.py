@@ -94,8 +94,9 @@ class ResidentInputs:
 class Job:
     """One context and the launch sequence of a whole pass."""
 
-    def __init__(self, w: synth.Workload, device, per_layer_decode=False, keep_steps=None):
+    def __init__(self, w: synth.Workload, device, per_layer_decode=False, keep_steps=None, exchange=None):
         self.w = w
+        self.exchange = exchange  # called with the context after the importance pass (one batch sharded over ranks)
         self.device = torch.device(device)
         self.ctx = context_for(w, device)
         self.per_layer_decode = per_layer_decode
@@ -110,6 +111,8 @@ class Job:
             a, b = inp.hidden[l]
             for _ in range(inp.hidden_repeat):
                 ctx.layer_importance(l, a, b)
+        if self.exchange is not None:
+            self.exchange(ctx)  # a batch sharded over ranks: the layer sums of all ranks, once, before the allocation
         ctx.allocate_budgets(w.b_init, w.p)
         for l in range(w.n_layer):
             q, k, v = inp.prompt(l)

@@ -50,6 +50,52 @@ def test_aggregate_throughput_two_ranks():
         assert mx == 1.0
 
 
+class _FakeCtx:
+    """Stands in for a context of one rank: holds the per-layer cosine sums and token counts that
+    rank accumulated over its share of the batch."""
+
+    def __init__(self, sums, counts):
+        self.sums, self.counts = list(sums), list(counts)
+
+    def get_importance_state(self):
+        return list(self.sums), list(self.counts)
+
+    def set_importance_state(self, sums, counts):
+        self.sums, self.counts = list(sums), list(counts)
+
+
+def _exchange_worker(rank, world, port, q):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    from paper_2404_04793_b200 import dist_util
+    dist_util.init("gloo")
+    # rank r holds 3 + r sequences of 100 tokens; three layers
+    ctx = _FakeCtx([10.0 + rank, 20.5 * (rank + 1), 0.125], [(3 + rank) * 100] * 3)
+    dist_util.exchange_importance(ctx)
+    dist_util.barrier()
+    dist_util.shutdown()
+    q.put((rank, ctx.sums, ctx.counts))
+
+
+def test_importance_exchange_of_a_batch_sharded_over_two_ranks():
+    """The one exchange of the path: the per-layer cosine sums and token counts of a batch whose
+    sequences are spread over the ranks are summed over all ranks, and every rank ends up with
+    the same totals (then the allocator, deterministic, gives every rank the same budgets)."""
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_exchange_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = [q.get(timeout=120) for _ in procs]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, sums, counts in res:
+        assert sums == [21.0, 61.5, 0.25]
+        assert counts == [700, 700, 700]
+
+
 def test_single_process_helpers_need_no_group():
     from paper_2404_04793_b200 import dist_util
     assert dist_util.max_over_ranks(3.5) == 3.5

@@ -79,6 +79,42 @@ def test_fused_importance_matches_oracle_and_the_two_call_form(dtype, hidden, ba
     assert fused.status() == 0
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_importance_state_exchange_gives_the_batch_budgets(dtype):
+    """A batch sharded over two ranks (emulated by two contexts, each fed half the sequences):
+    after the per-layer cosine sums and token counts are summed and put back, both allocate the
+    budgets the oracle derives from the whole batch's layer averages, and so does a context that
+    saw the whole batch."""
+    w = small("shard", 13, n_layer=6, hidden=512, batch=4, prompt=96, dtype=dtype)
+    whole = H.make_ctx(w)
+    whole.begin_sequence_batch(w.batch, w.prompt)
+    half = [H.make_ctx(w.replace(batch=2)) for _ in range(2)]
+    for h in half:
+        h.begin_sequence_batch(2, w.prompt)
+    cos_rows = []
+    for l in range(w.n_layer):
+        a, b = synth.hidden_pair(w, l, DEV)                      # [batch, prompt, hidden]
+        whole.layer_importance(l, a, b)
+        for r, h in enumerate(half):
+            h.layer_importance(l, a[2 * r:2 * r + 2].contiguous(), b[2 * r:2 * r + 2].contiguous())
+        cos_rows.append(O.layer_importance(H.f64(a).reshape(-1, w.hidden), H.f64(b).reshape(-1, w.hidden)))
+    states = [h.get_importance_state() for h in half]
+    sums = [x + y for x, y in zip(states[0][0], states[1][0])]
+    counts = [x + y for x, y in zip(states[0][1], states[1][1])]
+    assert counts == [w.batch * w.prompt] * w.n_layer
+    for h in half:
+        h.set_importance_state(sums, counts)
+        h.allocate_budgets(w.b_init, w.p)
+    whole.allocate_budgets(w.b_init, w.p)
+    cos = half[0].get_cos_sim().numpy().astype(np.float64)
+    assert np.max(np.abs(cos - np.array(cos_rows))) <= H.TOL_OUT[dtype]
+    assert np.max(np.abs(cos - whole.get_cos_sim().numpy().astype(np.float64))) <= 1e-6
+    want_b, want_g = O.allocate_budgets(half[0].get_cos_sim().numpy(), w.b_init, w.p)
+    for c in (half[0], half[1], whole):
+        assert c.get_budgets() == (want_b.tolist(), want_g.tolist())
+        assert c.status() == 0
+
+
 def test_layer_importance_special_vectors():
     w = small("imp2", 12, n_layer=4, hidden=64, batch=1, prompt=8)
     ctx = H.make_ctx(w)
