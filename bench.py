@@ -155,16 +155,19 @@ def _one_thread():
 
 
 def oracle_unit_task(task):
-    """One (layer, sequence, KV head) unit through the oracle: prompt, then every decode step.
-    Returns the seconds it took.  Runs in this process or in a worker of the all-cores pool."""
+    """One (layer, sequence, KV head) unit through the oracle: prompt, then its decode steps.
+    Returns the seconds it took, the decode steps scaled to the trajectory's full length when only
+    its first steps were sampled.  Runs in this process or in a worker of the all-cores pool."""
     from oracle import sq_oracle as O
     with _one_thread():
         t0 = time.perf_counter()
         u = O.UnitCache(task["policy"], task["budget"], task["n_sink"], task["heavy_num"], task["heavy_den"])
         u.prefill(task["k"], task["v"], task["q"])
+        t1 = time.perf_counter()
         for (q, kn, vn) in task["steps"]:
             u.decode_step(q, kn, vn)
-        return time.perf_counter() - t0
+        t2 = time.perf_counter()
+        return (t1 - t0) + (t2 - t1) * task.get("steps_scale", 1.0)
 
 
 def oracle_importance_task(task):
@@ -175,10 +178,12 @@ def oracle_importance_task(task):
         return time.perf_counter() - t0, c
 
 
-def oracle_tasks(w, n_units, n_imp_tokens, seed, device):
+def oracle_tasks(w, n_units, n_imp_tokens, seed, device, max_steps=None):
     """Draws a bounded sample of the workload for the oracle: importance chunks (a few layers,
-    n_imp_tokens tokens in all) and n_units (layer, sequence, KV head) units with all their decode
-    steps.  Returns (importance tasks, unit tasks, budgets)."""
+    n_imp_tokens tokens in all) and n_units (layer, sequence, KV head) units with their decode
+    steps: all of them, or the first max_steps when every sampled cache already holds its budget
+    after the prompt (a decode step then costs the same all along, and the unit's decode time is
+    scaled to the full trajectory).  Returns (importance tasks, unit tasks, budgets, steps sampled)."""
     import torch
     from oracle import sq_oracle as O
     from paper_2404_04793_b200 import synth
@@ -213,13 +218,18 @@ def oracle_tasks(w, n_units, n_imp_tokens, seed, device):
                           "n_sink": w.n_sink, "heavy_num": w.heavy_num, "heavy_den": w.heavy_den, "k": f64(k[s, h]),
                           "v": f64(v[s, h]), "q": None if q is None else f64(q[s, h * g:(h + 1) * g]), "steps": []})
         del q, k, v
-    for t in range(w.steps):
+    n_steps = w.steps
+    if max_steps and max_steps < w.steps and all(u["budget"] <= w.prompt for u in units):
+        n_steps = max_steps
+    for t in range(n_steps):
         dq, dk, dv = synth.decode_qkv(w, t, device)
         for u in units:
             l, s, h = u["layer"], u["seq"], u["head"]
             u["steps"].append((f64(dq[l, s, h * g:(h + 1) * g]), f64(dk[l, s, h]), f64(dv[l, s, h])))
         del dq, dk, dv
-    return imp, units, budgets
+    for u in units:
+        u["steps_scale"] = w.steps / n_steps
+    return imp, units, budgets, n_steps
 
 
 def extrapolate(w, budgets, imp_s_per_token, alloc_s, unit_s_by_layer):
@@ -234,7 +244,7 @@ def extrapolate(w, budgets, imp_s_per_token, alloc_s, unit_s_by_layer):
         + sum(unit_cost(l) * w.batch * w.n_kv_head for l in range(w.n_layer))
 
 
-def oracle_sample(w, n_units, n_imp_tokens, seed, device, pool_cores=0):
+def oracle_sample(w, n_units, n_imp_tokens, seed, device, pool_cores=0, max_steps=None):
     """Times the oracle on a bounded sample of the workload and extrapolates linearly to the
     whole job.  One thread in this process; with pool_cores > 1 the same kind of sample, pool_cores
     times as large, is then also run as a plain parallel-for over that many worker processes.
@@ -243,7 +253,7 @@ def oracle_sample(w, n_units, n_imp_tokens, seed, device, pool_cores=0):
     from oracle import sq_oracle as O
     t_start = time.perf_counter()
     n_total = n_units * max(1, pool_cores)
-    imp, units, budgets = oracle_tasks(w, n_total, n_imp_tokens * max(1, pool_cores), seed, device)
+    imp, units, budgets, n_steps = oracle_tasks(w, n_total, n_imp_tokens * max(1, pool_cores), seed, device, max_steps)
     # ---- one core: the first n_units-worth of the sample (spread over the layers) ----
     stride = max(1, len(units) // max(1, n_units))
     mine = units[::stride][:n_units]
@@ -266,7 +276,10 @@ def oracle_sample(w, n_units, n_imp_tokens, seed, device, pool_cores=0):
     t_job = extrapolate(w, budgets, t_imp / max(n_imp, 1), t_alloc, unit_s)
     total_units = w.n_layer * w.batch * w.n_kv_head
     out = {"value": w.batch * w.steps / t_job, "unit": UNIT, "cores": 1, "kind": "oracle",
-           "sample": (f"{len(mine)} (layer,seq,kv-head) units over {len(unit_s)} layers, all {w.steps} decode steps, "
+           "sample": (f"{len(mine)} (layer,seq,kv-head) units over {len(unit_s)} layers, "
+                      + (f"all {w.steps} decode steps, " if n_steps == w.steps else
+                         f"the first {n_steps} of {w.steps} decode steps (full caches: scaled to all steps), ")
+                      +
                       f"+ {n_imp} tokens of layer importance + the allocator; extrapolated linearly to "
                       f"{total_units} units and {w.n_layer * w.batch * w.prompt} tokens"),
            "job_seconds_extrapolated": t_job}
@@ -317,7 +330,8 @@ def run_reference(args, w):
     vals, secs = [], []
     desc = ""
     for i in range(args.warmup + args.steps):
-        r = oracle_sample(w, n_units=2, n_imp_tokens=2048, seed=100 + i, device=device)
+        # a quarter of the trajectory per sample keeps the default --steps 5 --warmup 3 run near two minutes
+        r = oracle_sample(w, n_units=2, n_imp_tokens=2048, seed=100 + i, device=device, max_steps=max(8, w.steps // 4))
         if i >= args.warmup:
             vals.append(r["value"]); secs.append(r["seconds"])
         desc = r["sample"]
