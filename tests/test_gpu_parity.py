@@ -113,6 +113,15 @@ def test_importance_state_exchange_gives_the_batch_budgets(dtype):
     for c in (half[0], half[1], whole):
         assert c.get_budgets() == (want_b.tolist(), want_g.tolist())
         assert c.status() == 0
+    # argument and mode errors: a count below 1; per-sequence budgets have nothing to exchange
+    with pytest.raises(B.SqError) as e:
+        half[0].set_importance_state(sums, [0] * w.n_layer)
+    assert e.value.code == B.SQ_ERR_INVALID_ARG
+    per_seq = H.make_ctx(w, per_sequence_budgets=1)
+    per_seq.begin_sequence_batch(w.batch, w.prompt)
+    with pytest.raises(B.SqError) as e:
+        per_seq.get_importance_state()
+    assert e.value.code == B.SQ_ERR_UNSUPPORTED
 
 
 def test_layer_importance_special_vectors():
