@@ -105,7 +105,10 @@ def decode_step_time(w: synth.Workload, steps=12, warmup=3, per_layer=False, dev
         with torch.cuda.graph(graph):
             for _ in range(steps):
                 step()
-        graph.replay()
+        if w.policy != synth.H2O:
+            graph.replay()
+        # (H2O: the captured steps carry their token positions, so a second replay would hand the
+        # score pass positions that run backwards; the first replay is the one that is timed)
         torch.cuda.synchronize()
         e0.record()
         graph.replay()
