@@ -9,7 +9,9 @@
 //   warp 1      MMA issue (one thread)
 //   warps 2..5  thread = one head row (TMEM lane): p = exp2(s*scale - m_ref) straight from the
 //               accumulator row, no shuffles; P is packed to bf16 and stored back to tensor
-//               memory as the A operand of the second MMA
+//               memory as the A operand of the second MMA.  A quarter of tensor memory with at
+//               most 8 head rows (g = 71: the third) is worked by its warp in quads instead, four
+//               threads to a row (sq_tc_quad.cuh)
 // Measured on B200: one M=128, K=16 MMA costs 45-48 cycles for N <= 64 and 64 cycles for N = 128,
 // and operands read from shared memory compete with the TMA writes for its 128 B/clk; keeping P
 // in tensor memory (64 columns) removes 56 KB of shared-memory traffic per tile.  Inside the
@@ -33,6 +35,7 @@
 #include "sq_decode_common.cuh"
 #include "sq_internal.h"
 #include "sq_tc.cuh"
+#include "sq_tc_quad.cuh"
 
 namespace sq {
 
@@ -52,6 +55,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+
 }  // namespace
 
 // ROWS: head rows of Q held in shared memory (96 or 128).
@@ -218,6 +222,17 @@ __global__ void __launch_bounds__(192, 2)
                    o_addr = tmem_base + lane_sel + kColO;
     float m_ref = -INFINITY, l = 0.f, l_w = 0.f;  // the row's reference; sums of its weights, exact and as rounded to bf16
     bool ok = true;
+    // quad form (see QuadCtx): m_ref is the row's (equal in its four threads), l and l_w are the
+    // thread's part; the row's totals are formed once, at the end
+    const int rows_here = G - quarter * 32;
+    const bool quad = rows_here >= 1 && rows_here <= 8 && n_tiles >= 6;  // short items: the set-up would not pay
+    const QuadCtx qc{s_addr, p_addr, bar_sfree, a.scale_log2, lane};
+    auto quad_sum = [&](float v) {
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      return v + __shfl_xor_sync(0xffffffffu, v, 2);
+    };
+    // the value the quad of row `lane` holds, for the lanes that own a row of O (others: their own)
+    auto from_row_quad = [&](float v) { return __shfl_sync(0xffffffffu, v, lane < 8 ? lane * 4 : lane); };
 
     // Row maximum of the tile's valid tokens, in the log2 domain.
     auto tile_max = [&](int n_valid) {
@@ -328,9 +343,27 @@ __global__ void __launch_bounds__(192, 2)
       tc_fence_after();
       bool s_released = false;
       if (warp_live) {
-        if (i == 0) m_ref = tile_max(n_valid);
+        if (i == 0) {
+          m_ref = quad ? quad_tile_max(qc, n_valid) : tile_max(n_valid);
+          if (quad) {
+            // rows 80..95 of P are never written in the quad form: clear them once
+            float z[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = 0.f;
+            tmem_st32(p_addr, z);
+            tmem_st32(p_addr + 32, z);
+          }
+        }
         float sum, sum_w;
         auto weights = [&]() {
+          if (quad) {
+            float sums[2];
+            s_released = (n_valid == kTM) ? quad_tile_weights<H2O, true, true>(qc, m_ref, n_valid, sums)
+                                          : quad_tile_weights<H2O, false, true>(qc, m_ref, n_valid, sums);
+            sum = sums[0];
+            sum_w = sums[1];
+            return sum_w;
+          }
           return (n_valid == kTM) ? tile_weights(std::true_type{}, n_valid, &sum, &sum_w, &s_released)
                                   : tile_weights(std::false_type{}, n_valid, &sum, &sum_w, &s_released);
         };
@@ -339,18 +372,25 @@ __global__ void __launch_bounds__(192, 2)
           // rare: move the reference of the rows that need it; O and the sums (complete up to
           // tile i-1) shrink with it, then the tile is redone.  The whole warp takes part in
           // the TMEM round trip.
-          const float mx2 = tile_max(n_valid);
-          const bool need = pmax > kMaxWeight;
+          const float mx2 = quad ? quad_tile_max(qc, n_valid) : tile_max(n_valid);
+          // quad form: the row moves when any of its four threads needs it
+          const bool need = quad ? __any_sync(0xfu << (lane & 28), pmax > kMaxWeight) : pmax > kMaxWeight;
           ok = mbar_wait(bar_odone, (i - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_ref - mx2) : 1.f;
+          // O is held a row per lane in either form
+          float f_o = f;
+          if (quad) {
+            f_o = from_row_quad(f);
+            if (lane >= 8) f_o = 1.f;
+          }
 #pragma unroll 1
           for (int c = 0; c < 2; ++c) {
             float o[32];
             tmem_ld32(o_addr + c * 32, o);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] *= f;
+            for (int j = 0; j < 32; ++j) o[j] *= f_o;
             tmem_st32(o_addr + c * 32, o);
           }
           l *= f;
@@ -375,6 +415,12 @@ __global__ void __launch_bounds__(192, 2)
       bf16* ob = reinterpret_cast<bf16*>(a.out) + (tok * a.n_q_head + (size_t)kvh * G) * kD;
       float* stat = a.part_stat + (size_t)blockIdx.x * G * kStatStride;
       float* po = a.part_o + (size_t)blockIdx.x * G * kD;
+      if (quad) {
+        // the row's totals from its four threads, then to the lane that holds the row of O
+        l = from_row_quad(quad_sum(l));
+        l_w = from_row_quad(quad_sum(l_w));
+        m_ref = from_row_quad(m_ref);
+      }
       const float inv = 1.f / l_w;
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
