@@ -12,20 +12,24 @@
 
 namespace sq {
 
-// One CTA (4 warps) per (layer, unit, split).  A K or V row is D*sizeof(T) bytes = LPR lanes
+// One CTA (NW warps) per (layer, unit, split).  A K or V row is D*sizeof(T) bytes = LPR lanes
 // x 16 bytes, so a warp reads 32/LPR consecutive rows per load instruction, fully coalesced.
 // Each lane keeps its 16-byte slice of up to GT query heads (pre-scaled by log2(e)/sqrt(d))
 // and of their output accumulators in fp32; logits are reduced over the LPR lanes by
 // shuffles, and the softmax runs online in the log2 domain over batches of U rows.
 // UNIFORM: the launch has no split-K (see locate()).
-template <typename T, int D, int GT, int UNIFORM, class Args>
-__global__ void __launch_bounds__(128, GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) decode_attn_kernel(Args a) {
+// NW = 4 everywhere but in the build for launches of few, unsplit units (one layer of a small
+// batch): those leave most warp slots of the GPU empty with 4 warps per unit, and each warp then
+// walks its rows in a chain of dependent round trips to memory; 16 warps per unit make the chain
+// a quarter as long.
+template <typename T, int D, int GT, int UNIFORM, class Args, int NW = 4>
+__global__ void __launch_bounds__(NW * 32, NW == 4 ? (GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) : 2) decode_attn_kernel(Args a) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;   // lanes per row
   constexpr int RPW = 32 / LPR;  // rows per warp per load
   constexpr int U = 4;           // rows in flight per lane
-  __shared__ float sm_o[4][GT][D];
-  __shared__ float sm_m[4][GT], sm_l[4][GT];
+  __shared__ float sm_o[NW][GT][D];
+  __shared__ float sm_m[NW][GT], sm_l[NW][GT];
 
   ItemLoc it;
   if (!locate<UNIFORM, Args>(a, blockIdx.x, it)) return;
@@ -77,7 +81,7 @@ __global__ void __launch_bounds__(128, GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) dec
         o[g][e] = 0.f;
       }
     }
-    for (int r0 = t0 + warp * (U * RPW); r0 < t1; r0 += 4 * U * RPW) {
+    for (int r0 = t0 + warp * (U * RPW); r0 < t1; r0 += NW * U * RPW) {
       uint4 kq[U], vq[U];
       bool ok[U];
 #pragma unroll
@@ -174,15 +178,15 @@ __global__ void __launch_bounds__(128, GT == 1 ? (UNIFORM == 1 ? 8 : 6) : 1) dec
       }
     }
     __syncthreads();
-    for (int idx = tid; idx < GT * D; idx += 128) {
+    for (int idx = tid; idx < GT * D; idx += NW * 32) {
       const int g = idx / D, e = idx - g * D, h = hb + g;
       if (h >= a.group) continue;
       float M = -INFINITY;
 #pragma unroll
-      for (int ww = 0; ww < 4; ++ww) M = fmaxf(M, sm_m[ww][g]);
+      for (int ww = 0; ww < NW; ++ww) M = fmaxf(M, sm_m[ww][g]);
       float L = 0.f, O = 0.f;
 #pragma unroll
-      for (int ww = 0; ww < 4; ++ww) {
+      for (int ww = 0; ww < NW; ++ww) {
         const float mw = sm_m[ww][g];
         const float f = (mw > -INFINITY) ? exp2f(mw - M) : 0.f;
         L += sm_l[ww][g] * f;
@@ -446,7 +450,9 @@ template <typename T, int D>
 static void launch_attn_g(const DecodeArgs& a, int n_items, cudaStream_t s) {
   if (a.group == 1) {
     // the register-capped kernel gets its own build for launches without split-K
-    if (a.uniform) decode_attn_kernel<T, D, 1, 1, DecodeArgsBase><<<n_items, 128, 0, s>>>(a);  // sliced: no table
+    // few unsplit units (at most two 16-warp CTAs per SM, all resident at once): 16 warps per unit
+    if (a.uniform && n_items <= 2 * 148) decode_attn_kernel<T, D, 1, 1, DecodeArgsBase, 16><<<n_items, 512, 0, s>>>(a);
+    else if (a.uniform) decode_attn_kernel<T, D, 1, 1, DecodeArgsBase><<<n_items, 128, 0, s>>>(a);  // sliced: no table
     else decode_attn_kernel<T, D, 1, 0, DecodeArgs><<<n_items, 128, 0, s>>>(a);
   } else if (a.group <= 4) {
     decode_attn_kernel<T, D, 4, -1, DecodeArgs><<<n_items, 128, 0, s>>>(a);

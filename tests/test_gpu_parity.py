@@ -332,6 +332,20 @@ def test_decode_per_layer_calls_and_growth_through_budget(policy):
     _run_decode_and_compare(w, budgets=[23, 6, 64], per_layer_calls=True)
 
 
+@pytest.mark.parametrize("policy", [synth.SLIDING_WINDOW, synth.STREAMING_LLM, synth.H2O])
+@pytest.mark.parametrize("dtype,head_dim", [(torch.bfloat16, 128), (torch.bfloat16, 64), (torch.float32, 128),
+                                            (torch.float32, 64)])
+def test_decode_one_head_per_kv_head_few_unsplit_units(policy, dtype, head_dim):
+    """One query head per KV head, few units, budgets short enough to stay unsplit: the launches
+    that give every unit 16 warps.  The budgets take a warp through one to five loads with a ragged
+    last one (a pass of the 16 warps covers 64 to 256 rows, by row size), called layer by layer
+    and for all layers at once."""
+    w = small("mha_few", 41, policy=policy, dtype=dtype, head_dim=head_dim, n_q_head=3, n_kv_head=3, batch=2,
+              n_layer=3, prompt=330, steps=4, heavy_mode="zipf")
+    _run_decode_and_compare(w, budgets=[277, 131, 65], per_layer_calls=True)
+    _run_decode_and_compare(w.replace(wid=42), budgets=[200, 290, 129])
+
+
 @pytest.mark.parametrize("policy", [synth.SLIDING_WINDOW, synth.H2O])
 def test_decode_split_k_long_context(policy):
     # few units, long budgets: the launch splits each unit's tokens over several CTAs
