@@ -698,6 +698,12 @@ def main():
     ap.add_argument("--no-records", action="store_true", help="skip the decode-step records of the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.impl == "ours" and args.gpus > 1 and "RANK" not in os.environ:
+        import torch
+        if torch.cuda.device_count() < args.gpus:
+            print(f"bench.py: --gpus {args.gpus} needs {args.gpus} CUDA devices, found {torch.cuda.device_count()}",
+                  file=sys.stderr)
+            sys.exit(2)
     rc = maybe_spawn(sys.argv[1:], args.gpus)
     if rc is not None:
         sys.exit(rc)
